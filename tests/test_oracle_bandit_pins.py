@@ -1,0 +1,192 @@
+"""Pins of the CPU oracle's bandit policies (MetaSD-UCB, Discounted UCB, Sliding-window UCB).
+
+Expected values are invariants, textbook consequences of the index rule, the explicit-constant
+pull bound the paper quotes, and reductions between the variants -- never the oracle's own output.
+"""
+import math
+
+import numpy as np
+import pytest
+
+from oracle import oracle as O
+
+
+def run_bandit(variant, K, reward_fn, rounds, beta=1.0, gamma=1.0, tau=10 ** 6, seed=0):
+    """Drive one oracle bandit instance with rewards reward_fn(arm, t, rng); returns the logs."""
+    cfg = O.OracleConfig(max_batch=1, n_drafters=K, vocab=1, bandit=variant, beta=beta, gamma=gamma,
+                         tau=min(tau, rounds + 1))
+    orc = O.OracleMetaSD(cfg)
+    rng = np.random.RandomState(seed)
+    arms, rewards = [], []
+    for t in range(rounds):
+        a = int(orc.select()[0])
+        r = float(reward_fn(a, t, rng))
+        orc.update([a], [r])
+        arms.append(a)
+        rewards.append(r)
+    return np.array(arms), np.array(rewards), orc
+
+
+def test_init_sweep_plays_every_arm_once_in_order():
+    for variant in (O.UCB, O.DUCB, O.SWUCB):
+        arms, _, orc = run_bandit(variant, 5, lambda a, t, g: g.rand(), 5, gamma=0.9, tau=50)
+        assert arms.tolist() == [0, 1, 2, 3, 4]
+        assert orc.t[0] == 5
+    arms, _, _ = run_bandit(O.UCB, 1, lambda a, t, g: g.rand(), 20)      # K = 1: ln 1 = 0, always arm 0
+    assert (arms == 0).all()
+
+
+def test_ucb_mean_is_the_batch_mean_and_counts_are_pull_counts():
+    arms, rewards, orc = run_bandit(O.UCB, 4, lambda a, t, g: g.beta(1 + a, 2), 400, beta=0.5, seed=3)
+    mu, n = orc.mean_estimates()
+    for i in range(4):
+        assert n[0, i] == (arms == i).sum()
+        assert abs(mu[0, i] - rewards[arms == i].mean()) < 1e-12
+    assert n.sum() == 400
+
+
+def test_equal_means_make_ucb_round_robin():
+    """With identical constant rewards the index differs only by sqrt(2 ln t / n_i): the least
+    pulled arm wins, lowest index first, so the arms are played in strict rotation."""
+    arms, _, _ = run_bandit(O.UCB, 4, lambda a, t, g: 0.5, 80, beta=0.3)
+    assert arms.tolist() == [t % 4 for t in range(80)]
+
+
+def test_zero_exploration_is_greedy_on_the_means():
+    means = [0.2, 0.7, 0.4]
+    arms, _, _ = run_bandit(O.UCB, 3, lambda a, t, g: means[a], 50, beta=0.0)
+    assert arms[:3].tolist() == [0, 1, 2] and (arms[3:] == 1).all()
+
+
+@pytest.mark.parametrize("beta,delta,T", [(1.0, 0.5, 20000), (0.5, 0.3, 20000), (1.0, 0.25, 50000)])
+def test_deterministic_two_arm_pull_count_matches_index_equalisation(beta, delta, T):
+    """Two arms with constant rewards c0 > c1.  UCB keeps the two indices level, so after T rounds
+    the worse arm's count n1 solves c1 + beta sqrt(2 ln T / n1) = c0 + beta sqrt(2 ln T / (T - n1)).
+    This fixes the constant 2, the natural logarithm and beta in the exploration term."""
+    c0, c1 = 0.8, 0.8 - delta
+    arms, _, _ = run_bandit(O.UCB, 2, lambda a, t, g: (c0, c1)[a], T, beta=beta)
+    n1 = int((arms == 1).sum())
+    L = 2.0 * math.log(T)
+    x = 1.0
+    for _ in range(200):                              # fixed point of the level-index equation
+        x = beta ** 2 * L / (delta + beta * math.sqrt(L / (T - x))) ** 2
+    assert abs(n1 - x) <= 0.05 * x + 2, (n1, x)
+    # a missing factor 2, log10 or log2 instead of ln would be far outside this band
+    assert abs(x / 2 - n1) > 0.2 * x and abs(x / math.log(10) - n1) > 0.2 * x
+
+
+def test_suboptimal_pull_bound_with_explicit_constants():
+    """E[n_i(tau)] <= 8 ln tau / Delta_i^2 + 1 + pi^2/3 for beta = 1 (the lemma quoted from Auer et al.)."""
+    means = np.array([0.75, 0.55, 0.35])
+    rounds, seeds = 3000, 60
+    pulls = np.zeros((seeds, 3))
+    for s in range(seeds):
+        arms, _, _ = run_bandit(O.UCB, 3, lambda a, t, g: g.beta(4 * means[a], 4 * (1 - means[a])), rounds,
+                                beta=1.0, seed=s)
+        pulls[s] = np.bincount(arms, minlength=3)
+    for i in (1, 2):
+        delta = means[0] - means[i]
+        bound = 8 * math.log(rounds) / delta ** 2 + 1 + math.pi ** 2 / 3
+        assert pulls[:, i].mean() <= bound
+    assert pulls[:, 0].mean() > 0.6 * rounds            # the best arm dominates
+    # the number of suboptimal pulls grows like ln(rounds), not linearly: x10 rounds -> far less than x10 pulls
+    short = np.mean([np.bincount(run_bandit(O.UCB, 3, lambda a, t, g: g.beta(4 * means[a], 4 * (1 - means[a])),
+                                            300, beta=1.0, seed=s)[0], minlength=3)[1:].sum() for s in range(30)])
+    assert pulls[:, 1:].sum(axis=1).mean() < 4.0 * short
+
+
+def test_bd_form_of_the_pull_bound():
+    """With the BD reward (mean of N_max i.i.d. alignment samples) and beta = 1/sqrt(N_max) the
+    bound tightens to 8 ln tau / (N_max Delta^2) + 1 + pi^2/3."""
+    k = 5
+    alphas = np.array([0.8, 0.6])
+    rounds, seeds = 3000, 60
+    pulls = []
+    for s in range(seeds):
+        arms, _, _ = run_bandit(
+            O.UCB, 2, lambda a, t, g: g.beta(4 * alphas[a], 4 * (1 - alphas[a]), size=k).mean(), rounds,
+            beta=1 / math.sqrt(k), seed=1000 + s)
+        pulls.append((arms == 1).sum())
+    bound = 8 * math.log(rounds) / (k * 0.2 ** 2) + 1 + math.pi ** 2 / 3
+    assert np.mean(pulls) <= bound
+
+
+def test_ducb_and_swucb_reduce_to_ucb():
+    """gamma = 1 and a window longer than the run reproduce Algorithm 2 arm for arm."""
+    fn = lambda a, t, g: g.beta(2 + a, 3)
+    for beta in (0.01, 0.4, 1.0):
+        base, rew, _ = run_bandit(O.UCB, 5, fn, 600, beta=beta, seed=11)
+        d_arms, d_rew, _ = run_bandit(O.DUCB, 5, fn, 600, beta=beta, gamma=1.0, seed=11)
+        s_arms, s_rew, _ = run_bandit(O.SWUCB, 5, fn, 600, beta=beta, tau=10 ** 6, seed=11)
+        assert d_arms.tolist() == base.tolist() and np.array_equal(d_rew, rew)
+        assert s_arms.tolist() == base.tolist() and np.array_equal(s_rew, rew)
+
+
+def test_ducb_recursion_equals_the_direct_discounted_sums():
+    gamma = 0.93
+    arms, rewards, orc = run_bandit(O.DUCB, 4, lambda a, t, g: g.rand(), 300, beta=0.2, gamma=gamma, seed=5)
+    t_end = len(arms)
+    w = gamma ** (t_end - 1 - np.arange(t_end))        # weight of round s once round t_end-1 is in
+    mu, n = orc.mean_estimates()
+    for i in range(4):
+        S = (w * rewards * (arms == i)).sum()
+        N = (w * (arms == i)).sum()
+        assert abs(n[0, i] - N) < 1e-10 and abs(mu[0, i] - S / N) < 1e-10
+
+
+def test_swucb_window_holds_exactly_the_last_tau_rounds():
+    tau = 17
+    arms, rewards, orc = run_bandit(O.SWUCB, 3, lambda a, t, g: g.rand(), 200, beta=0.3, tau=tau, seed=6)
+    mu, n = orc.mean_estimates()
+    last_a, last_r = arms[-tau:], rewards[-tau:]
+    for i in range(3):
+        assert n[0, i] == (last_a == i).sum()
+        if n[0, i] > 0:
+            assert abs(mu[0, i] - last_r[last_a == i].mean()) < 1e-12
+
+
+def test_swucb_arm_that_left_the_window_is_played_again():
+    """An arm with no pull inside the window has an infinite index (lowest index first)."""
+    means = [0.9, 0.1, 0.1]
+    arms, _, _ = run_bandit(O.SWUCB, 3, lambda a, t, g: means[a], 60, beta=0.01, tau=8)
+    # arm 0 is best, but every arm reappears at least once in any stretch of tau + 3 rounds
+    for start in range(3, 60 - 11):
+        assert set(arms[start:start + 11].tolist()) == {0, 1, 2}
+
+
+def test_nonstationary_variants_recover_after_a_swap():
+    """After the arm means swap, D-UCB and SW-UCB return to the new best arm; plain UCB lags."""
+    def fn(a, t, g):
+        means = (0.8, 0.5) if t < 1500 else (0.4, 0.5)
+        return g.beta(8 * means[a], 8 * (1 - means[a]))
+    ratio = {}
+    for name, variant, kw in (("ucb", O.UCB, {}), ("ducb", O.DUCB, dict(gamma=0.97)),
+                              ("sw", O.SWUCB, dict(tau=100))):
+        hits = []
+        for s in range(10):
+            arms, _, _ = run_bandit(variant, 2, fn, 2000, beta=0.1, seed=s, **kw)
+            hits.append((arms[1600:] == 1).mean())
+        ratio[name] = np.mean(hits)
+    assert ratio["ducb"] > 0.7 and ratio["sw"] > 0.8 and ratio["ucb"] < 0.2
+    
+
+def test_select_reports_the_index_gap():
+    stat_a = np.array([0.5, 0.4, 0.1])
+    stat_b = np.array([10.0, 10.0, 10.0])
+    a, gap = O.bandit_select(O.UCB, 3, 0.2, 1, 30, stat_a, stat_b)
+    assert a == 0 and abs(gap - 0.1) < 1e-12           # equal counts: the gap is the mean gap
+    a, gap = O.bandit_select(O.UCB, 3, 0.2, 1, 30, np.array([0.4, 0.4, 0.1]), stat_b)
+    assert a == 0 and gap == 0.0                         # exact tie: lowest index
+
+
+def test_first_selection_after_the_sweep_uses_ln_of_completed_rounds():
+    """Algorithm 2 increments t in the init loop, so the selection after t completed rounds uses ln t.
+    Hand case, K = 2, t = 3, mu_hat = (0.5, 0), n = (2, 1):
+      index_0 = 0.5 + beta sqrt(2 ln 3 / 2) = 0.5 + 1.04815 beta,  index_1 = beta sqrt(2 ln 3) = 1.48230 beta,
+    so arm 1 wins iff beta > 0.5 / 0.43415 = 1.1517.  (With ln(t+1) the boundary would be 1.0252,
+    with ln(t-1) it would be 1.4498.)"""
+    mu, n = np.array([0.5, 0.0]), np.array([2.0, 1.0])
+    assert O.bandit_select(O.UCB, 2, 1.10, 1, 3, mu, n)[0] == 0
+    assert O.bandit_select(O.UCB, 2, 1.14, 1, 3, mu, n)[0] == 0
+    assert O.bandit_select(O.UCB, 2, 1.16, 1, 3, mu, n)[0] == 1
+    assert O.bandit_select(O.UCB, 2, 1.40, 1, 3, mu, n)[0] == 1
