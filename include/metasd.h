@@ -1,0 +1,177 @@
+/*
+ * metasd.h -- C ABI of the MetaSD draft-verify hot path on NVIDIA B200 (sm_100a).
+ *
+ * One MetaSD round (Algorithm 1 of the paper: "meta-draft a drafter following the bandit ->
+ * one speculative-decoding step -> block-divergence reward -> update the bandit") for a batch of
+ * B independent sequences, each with its own bandit instance over K drafters:
+ *
+ *   metasd_select  : the drafter each sequence plays this round           (Algorithm 2, line 7)
+ *   metasd_verify  : speculative-sampling verification of k drafted tokens (Algorithm 4, lines 6-12),
+ *                    the alignment reward (Definition 2, Eq. 4; or block efficiency, Sec. 2.3),
+ *                    the bandit update (Algorithm 2, lines 9-10; Discounted UCB and Sliding-window
+ *                    UCB of the non-stationary appendix) and the next round's selection.
+ *
+ * Conventions
+ *   - Every pointer is a DEVICE pointer unless the parameter name starts with host_.
+ *   - Logit tensors are dense, row-major, innermost dimension V (the vocabulary).  Rows whose
+ *     byte length and base address are multiples of 16 take the vectorised path; anything else
+ *     is still correct through a scalar path.
+ *   - The caller owns every input and output buffer.  The library owns the context, the bandit
+ *     state and its scratch; nothing is allocated after metasd_init.
+ *   - Calls are asynchronous on the CUDA stream passed as `stream` (a cudaStream_t, typed void*
+ *     so that this header needs no CUDA include); calls on one context must be stream-ordered.
+ *   - Every function returns 0 (METASD_OK) or a negative metasd_error.  Device-side anomalies
+ *     never trap: they set bits in the context's status word and produce the defined outputs
+ *     described at metasd_last_status.
+ *   - There is no CPU fallback: without a CUDA device metasd_init fails with METASD_ERR_CUDA.
+ */
+#ifndef METASD_H
+#define METASD_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct metasd_ctx metasd_ctx;
+
+enum metasd_error {
+    METASD_OK = 0,
+    METASD_ERR_INVALID_ARGUMENT = -1,
+    METASD_ERR_UNSUPPORTED = -2,
+    METASD_ERR_CUDA = -3,
+    METASD_ERR_NO_MEMORY = -4,
+    METASD_ERR_BAD_STATE_BLOB = -5
+};
+
+enum metasd_dtype { METASD_BF16 = 0, METASD_FP32 = 1 };
+enum metasd_bandit { METASD_UCB = 0, METASD_DUCB = 1, METASD_SWUCB = 2 };
+enum metasd_reward { METASD_REWARD_BD = 0, METASD_REWARD_BE = 1 };
+
+/* Which kernels metasd_verify launches. */
+enum metasd_path {
+    METASD_PATH_AUTO = 0,      /* fused cluster kernel when the shape fits it, else streaming */
+    METASD_PATH_STREAMING = 1, /* row-statistics kernel + per-sequence epilogue kernel; any shape */
+    METASD_PATH_FUSED = 2      /* one persistent thread-block-cluster kernel per call */
+};
+
+/* Status bits (OR-accumulated on the device until read). */
+#define METASD_STATUS_NONFINITE 1u /* a row held NaN / +Inf or no finite entry */
+#define METASD_STATUS_TOKEN_OOR 2u /* a drafted token id was outside [0, V) */
+#define METASD_STATUS_Q_ZERO    4u /* the drafter gave probability 0 to its own drafted token */
+
+/* Hyper-parameters of metasd_init.  Paper notation: n_drafters = K, max_draft = N_max, beta = the
+ * exploration strength of Algorithm 2 (experiments: 0.01), gamma = the D-UCB decay, window = the
+ * SW-UCB window tau (neither value is given in the paper; 0.975 / 50 are this library's defaults). */
+typedef struct metasd_config {
+    int32_t max_batch;          /* B: sequences, 1 .. 65535 */
+    int32_t n_drafters;         /* K: 1 .. 16 */
+    int32_t max_draft;          /* N_max: 1 .. 16 */
+    int32_t vocab;              /* V >= 1 */
+    int32_t logit_dtype;        /* metasd_dtype */
+    int32_t bandit;             /* metasd_bandit */
+    int32_t reward;             /* metasd_reward */
+    int32_t window;             /* tau >= 1 (used by METASD_SWUCB) */
+    int32_t device;             /* CUDA device ordinal */
+    int32_t path;               /* metasd_path */
+    uint32_t sequence_base;     /* id of sequence 0 in the random-number key (batch sharding) */
+    int32_t host_staging;       /* != 0: also allocate device staging for metasd_verify_host */
+    double beta;
+    double gamma;
+    double reward_temperature;  /* softmax temperature of the reward when verifying greedily */
+} metasd_config;
+
+/* Optional per-position diagnostics of metasd_verify, [B, k]. */
+typedef struct metasd_diag {
+    float p_x;      /* target probability of the drafted token */
+    float q_x;      /* drafter probability of the drafted token */
+    float D;        /* d_TV(p_j, q_j) */
+    float u;        /* the uniform of the accept test */
+    int32_t accept; /* 1 = the accept test passed at this position */
+} metasd_diag;
+
+/* Fills *cfg with the defaults (UCB, BD reward, beta 0.01, gamma 0.975, window 50, bf16, auto path). */
+void metasd_default_config(metasd_config *cfg);
+
+/* Creates a context on cfg->device: validates cfg, allocates bandit state, scratch and (optionally)
+ * staging, and resets every sequence (Algorithm 2, line 1: t <- 0).  *out is NULL on failure. */
+int metasd_init(metasd_ctx **out, const metasd_config *cfg);
+
+/* Frees everything metasd_init allocated.  NULL is accepted. */
+void metasd_destroy(metasd_ctx *ctx);
+
+/* Per-query re-initialisation ("the bandit is re-initialised for every new query", experimental
+ * setup): t <- 0 and cleared arm statistics for the n sequences listed in seq_ids (device int32),
+ * or for all sequences when seq_ids is NULL.  Ids outside [0, max_batch) are ignored. */
+int metasd_reset(metasd_ctx *ctx, const int32_t *seq_ids, int32_t n, void *stream);
+
+/* Algorithm 2, lines 2-7: arm_out[b] = the drafter sequence b plays this round, b < batch.
+ * Rounds t < K play arm t (the initial sweep); afterwards argmax_i mu_i + beta sqrt(2 ln t / n_i),
+ * lowest index on ties; an arm with no pull inside the SW-UCB window scores +infinity. */
+int metasd_select(metasd_ctx *ctx, int32_t batch, int32_t *arm_out, void *stream);
+
+/* One verification round for sequences 0 .. batch-1 (Algorithm 4 lines 6-12, Definition 2,
+ * Algorithm 2 lines 9-10, then the next selection).
+ *
+ *   target_logits  [batch, k+1, V]  target logits at the k drafted positions and the bonus position
+ *   draft_logits   [batch, k, V]    the played drafter's logits, already gathered by arm; or NULL and
+ *   drafter_ptrs   device table of K pointers, each [batch, k, V]; the kernel reads table[arm[b]]
+ *   draft_tokens   [batch, k] int32 when token_arm_stride == 0, else [K, ...] with
+ *                  token_arm_stride int32 elements between consecutive drafters' [batch, k] blocks
+ *   temperature    T > 0: accept iff u < min(1, p(x)/q(x)) with p, q = softmax(logits / T);
+ *                  T == 0: greedy, accept iff x == argmax of the target row (lowest id on ties) and
+ *                  the reward uses softmax(logits / reward_temperature)
+ *   seed           key of the counter-based Philox4x32-10 stream; the counter is
+ *                  (sequence_base + b, round t of sequence b, position j, 0); word 0 drives the
+ *                  accept test, word 1 the residual / bonus draw; uniform = top 24 bits * 2^-24
+ *   accepted_len   [batch] int32, N_acc in [0, k]
+ *   next_token     [batch] int32, drawn from max(0, p - q) at the first rejection (inverse CDF in
+ *                  token order), or from p at position k if all accepted; greedy: the argmax;
+ *                  -1 when the row it needs is flagged non-finite
+ *   reward         [batch] fp32, BD: 1 - mean_j d_TV(p_j, q_j) over all k positions; BE: N_acc / k
+ *   diag           optional [batch, k]
+ *
+ * On return (stream order) each sequence's round counter is t+1 and its statistics include the
+ * reward.  Errors: invalid sizes / NULL pointers / both or neither draft source -> INVALID_ARGUMENT. */
+int metasd_verify(metasd_ctx *ctx, int32_t batch, int32_t k, const void *target_logits,
+                  const void *draft_logits, const void *const *drafter_ptrs,
+                  const int32_t *draft_tokens, int64_t token_arm_stride, float temperature,
+                  uint64_t seed, int32_t *accepted_len, int32_t *next_token, float *reward,
+                  metasd_diag *diag, void *stream);
+
+/* The same round with HOST buffers (gathered draft logits only): copies the inputs to the context's
+ * staging memory, runs metasd_verify, copies the three outputs (and host_arm_next, optional: the
+ * next round's selection) back, and synchronises the stream.  Needs cfg.host_staging != 0.
+ * Pinned host memory makes the copies asynchronous. */
+int metasd_verify_host(metasd_ctx *ctx, int32_t batch, int32_t k, const void *host_target_logits,
+                       const void *host_draft_logits, const int32_t *host_draft_tokens,
+                       float temperature, uint64_t seed, int32_t *host_accepted_len,
+                       int32_t *host_next_token, float *host_reward, int32_t *host_arm_next,
+                       void *stream);
+
+/* Bandit state as a flat blob in HOST memory (round counters, current arms, arm statistics,
+ * SW-UCB windows, and a header that import checks against the context's configuration).
+ * Both calls synchronise the stream. */
+size_t metasd_state_bytes(const metasd_ctx *ctx);
+int metasd_state_export(metasd_ctx *ctx, void *host_buf, size_t bytes, void *stream);
+int metasd_state_import(metasd_ctx *ctx, const void *host_buf, size_t bytes, void *stream);
+
+/* Reads and clears the status word (synchronises the stream).  Defined outputs: a non-finite row
+ * pair is rejected with d_TV = 1; an out-of-range token is rejected; q(x) = 0 < p(x) is accepted. */
+int metasd_last_status(metasd_ctx *ctx, uint32_t *host_flags, void *stream);
+
+/* Number of kernels this context has launched so far. */
+uint64_t metasd_kernel_launches(const metasd_ctx *ctx);
+
+/* The path metasd_verify takes for draft length k with the context's configuration
+ * (METASD_PATH_STREAMING or METASD_PATH_FUSED). */
+int metasd_resolved_path(const metasd_ctx *ctx, int32_t k);
+
+const char *metasd_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* METASD_H */

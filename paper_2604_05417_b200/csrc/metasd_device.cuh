@@ -1,0 +1,208 @@
+// Device-side building blocks of the MetaSD hot path: Philox4x32-10, fast exp2, 16-byte logit
+// vectors, warp/block reductions and the fp64 bandit arithmetic.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <math.h>
+#include <stdint.h>
+
+#include "metasd_internal.h"
+
+namespace metasd {
+
+// A finite stand-in for "no maximum yet": keeps (x - max) * c finite for masked (-inf) logits.
+#define METASD_NEG_BIG (-1.0e30f)
+
+// ---------------------------------------------------------------------------------------------
+// Philox4x32-10 (Salmon et al., SC'11): ten rounds of two 32x32->64 multiplies and key bumps.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint4 philox4x32_10(uint4 ctr, uint2 key)
+{
+    const uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u;
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        uint32_t hi0 = __umulhi(M0, ctr.x), lo0 = M0 * ctr.x;
+        uint32_t hi1 = __umulhi(M1, ctr.z), lo1 = M1 * ctr.z;
+        ctr = make_uint4(hi1 ^ ctr.y ^ key.x, lo1, hi0 ^ ctr.w ^ key.y, lo0);
+        key.x += 0x9E3779B9u;
+        key.y += 0xBB67AE85u;
+    }
+    return ctr;
+}
+
+// Uniform in [0, 1) from the top 24 bits of a word (exact in fp32).
+__device__ __forceinline__ float uniform24(uint32_t w) { return (float)(w >> 8) * (1.0f / 16777216.0f); }
+
+// The random words of (seed, sequence, round, position): .x accept test, .y residual / bonus draw.
+__device__ __forceinline__ uint4 round_words(uint64_t seed, uint32_t sequence, uint32_t round, uint32_t position)
+{
+    return philox4x32_10(make_uint4(sequence, round, position, 0u),
+                         make_uint2((uint32_t)(seed & 0xFFFFFFFFu), (uint32_t)(seed >> 32)));
+}
+
+// ---------------------------------------------------------------------------------------------
+// exp2 on the special-function unit (flushes denormals; relative error about 2^-22)
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ float ex2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Logit element types: 16-byte vectors of bf16 (8 per vector) or fp32 (4 per vector)
+// ---------------------------------------------------------------------------------------------
+template <typename LT> struct Logit;
+
+template <> struct Logit<__nv_bfloat16> {
+    static constexpr int VEC = 8;
+    __device__ static __forceinline__ void unpack(const uint4 &raw, float (&x)[8])
+    {
+        const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            x[2 * i] = __uint_as_float(w[i] << 16);
+            x[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+        }
+    }
+    __device__ static __forceinline__ float scalar(const __nv_bfloat16 *p, size_t i)
+    {
+        return __uint_as_float((uint32_t)reinterpret_cast<const uint16_t *>(p)[i] << 16);
+    }
+};
+
+template <> struct Logit<float> {
+    static constexpr int VEC = 4;
+    __device__ static __forceinline__ void unpack(const uint4 &raw, float (&x)[4])
+    {
+        x[0] = __uint_as_float(raw.x);
+        x[1] = __uint_as_float(raw.y);
+        x[2] = __uint_as_float(raw.z);
+        x[3] = __uint_as_float(raw.w);
+    }
+    __device__ static __forceinline__ float scalar(const float *p, size_t i) { return p[i]; }
+};
+
+// Streaming 16-byte load that does not allocate in L1.
+__device__ __forceinline__ uint4 ld_stream(const void *p)
+{
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Online softmax statistics relative to the raw maximum m: s = sum 2^((x - m) c)
+// ---------------------------------------------------------------------------------------------
+struct MaxSum {
+    float m, s;
+};
+
+__device__ __forceinline__ MaxSum merge(MaxSum a, MaxSum b, float c)
+{
+    MaxSum r;
+    r.m = fmaxf(a.m, b.m);
+    r.s = a.s * ex2((a.m - r.m) * c) + b.s * ex2((b.m - r.m) * c);
+    return r;
+}
+
+__device__ __forceinline__ MaxSum warp_merge(MaxSum v, float c)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        MaxSum w;
+        w.m = __shfl_xor_sync(0xFFFFFFFFu, v.m, o);
+        w.s = __shfl_xor_sync(0xFFFFFFFFu, v.s, o);
+        v = merge(v, w, c);
+    }
+    return v;
+}
+
+struct ArgMax {
+    float v;
+    int32_t i;
+};
+
+__device__ __forceinline__ ArgMax better(ArgMax a, ArgMax b)
+{
+    return (b.v > a.v || (b.v == a.v && b.i < a.i)) ? b : a;
+}
+
+__device__ __forceinline__ ArgMax warp_argmax(ArgMax a)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        ArgMax b;
+        b.v = __shfl_xor_sync(0xFFFFFFFFu, a.v, o);
+        b.i = __shfl_xor_sync(0xFFFFFFFFu, a.i, o);
+        a = better(a, b);
+    }
+    return a;
+}
+
+__device__ __forceinline__ double warp_sum(double v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    return v;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Bandit arithmetic in fp64 (Algorithm 2; Discounted UCB; Sliding-window UCB)
+// ---------------------------------------------------------------------------------------------
+// Arm for round t of one sequence.  sa/sb: this sequence's [K] statistics; wa/wr: its window.
+__device__ inline int bandit_select(int variant, int K, double beta, int tau, int t, const double *sa,
+                                    const double *sb, const int32_t *wa, const double *wr)
+{
+    if (t < K) return t;  // initial sweep: every drafter once, in order
+    double mu[16], n[16];
+    if (variant == METASD_SWUCB) {
+        for (int i = 0; i < K; ++i) { mu[i] = 0.0; n[i] = 0.0; }
+        int first = t - tau > 0 ? t - tau : 0;
+        for (int s = first; s < t; ++s) {  // oldest first
+            int slot = s % tau;
+            int i = wa[slot];
+            mu[i] += wr[slot];
+            n[i] += 1.0;
+        }
+        for (int i = 0; i < K; ++i)
+            if (n[i] > 0.0) mu[i] /= n[i];
+    } else if (variant == METASD_DUCB) {
+        for (int i = 0; i < K; ++i) { n[i] = sb[i]; mu[i] = sa[i] / sb[i]; }
+    } else {
+        for (int i = 0; i < K; ++i) { mu[i] = sa[i]; n[i] = sb[i]; }
+    }
+    const double two_ln_t = 2.0 * log((double)t);
+    int best = 0;
+    double best_score = -INFINITY;
+    for (int i = 0; i < K; ++i) {
+        double score = n[i] > 0.0 ? mu[i] + beta * sqrt(two_ln_t / n[i]) : INFINITY;
+        if (score > best_score) { best_score = score; best = i; }
+    }
+    return best;
+}
+
+// Folds reward r of arm a into the statistics and advances the round counter.
+__device__ inline void bandit_update(int variant, int K, double gamma, int tau, int32_t *t, double *sa,
+                                     double *sb, int32_t *wa, double *wr, int a, double r)
+{
+    if (variant == METASD_UCB) {
+        double n = sb[a];
+        sa[a] = (sa[a] * n + r) / (n + 1.0);
+        sb[a] = n + 1.0;
+    } else if (variant == METASD_DUCB) {
+        for (int i = 0; i < K; ++i) { sa[i] *= gamma; sb[i] *= gamma; }
+        sa[a] += r;
+        sb[a] += 1.0;
+    } else {
+        int slot = *t % tau;
+        wa[slot] = a;
+        wr[slot] = r;
+    }
+    *t = *t + 1;
+}
+
+}  // namespace metasd

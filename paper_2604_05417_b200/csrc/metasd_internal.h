@@ -1,0 +1,70 @@
+// Internal declarations shared by the translation units of libmetasd (not part of the C ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "metasd.h"
+
+namespace metasd {
+
+// Per-(sequence, position) result of the row-statistics pass; the scratch the streaming path keeps
+// between its two kernels.  Softmax terms are held relative to the raw row maximum:
+//   p_v = 2^((x_v - max_a) * c) / sum_a,  c = log2(e) / T.
+struct RowStats {
+    float max_a, sum_a;   // target row
+    float max_b, sum_b;   // draft row (unused at the bonus position)
+    double sum_min;       // sum_v min(p_v, q_v) = 1 - d_TV(p, q)
+    int32_t argmax_a;     // first index of the target row's maximum
+    uint32_t flags;       // METASD_STATUS_* of this row pair
+};
+
+// Bandit state of all sequences, structure of arrays in device memory.
+struct BanditState {
+    int32_t *t;          // [B] rounds completed
+    int32_t *arm;        // [B] arm to play in round t
+    double *stat_a;      // [B, K] UCB: mu_hat;  D-UCB: discounted reward sum
+    double *stat_b;      // [B, K] UCB: n;       D-UCB: discounted count
+    int32_t *win_arm;    // [B, tau] SW-UCB: arm of round s in slot s mod tau
+    double *win_reward;  // [B, tau]
+};
+
+struct VerifyParams {
+    // shapes
+    int32_t batch, k, V;
+    int32_t K, bandit, reward_kind, tau;
+    uint32_t sequence_base;
+    // inputs
+    const void *target;
+    const void *draft;                 // gathered, or nullptr
+    const void *const *drafter_ptrs;   // table, or nullptr
+    const int32_t *tokens;
+    int64_t token_arm_stride;
+    // math
+    float c;           // log2(e) / softmax temperature
+    int32_t greedy;
+    uint64_t seed;
+    double beta, gamma;
+    // outputs
+    int32_t *accepted_len;
+    int32_t *next_token;
+    float *reward;
+    metasd_diag *diag;
+    // state + scratch
+    BanditState st;
+    RowStats *stats;   // [batch, k+1]
+    uint32_t *status;
+    int32_t vector_ok; // rows are 16-byte aligned and a whole number of 16-byte vectors
+};
+
+// streaming path (metasd_streaming.cu)
+cudaError_t launch_streaming(const VerifyParams &p, int dtype, cudaStream_t stream, uint64_t *launches);
+// fused cluster path (metasd_fused.cu)
+bool fused_supported(int dtype, int V, int k);
+cudaError_t fused_prepare(int device);
+cudaError_t launch_fused(const VerifyParams &p, int dtype, cudaStream_t stream, uint64_t *launches);
+// small state kernels (metasd_streaming.cu)
+cudaError_t launch_select(const BanditState &st, int batch, int32_t *arm_out, cudaStream_t stream);
+cudaError_t launch_reset(const BanditState &st, int max_batch, int K, int tau, const int32_t *seq_ids,
+                         int n, cudaStream_t stream);
+
+}  // namespace metasd

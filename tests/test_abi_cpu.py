@@ -1,0 +1,91 @@
+"""CPU checks of the C-ABI library: it builds, loads, exports every declared symbol, validates
+arguments on the host, and fails loudly (no fallback) when there is no CUDA device."""
+import ctypes as C
+import os
+import re
+
+import pytest
+import torch
+
+from paper_2604_05417_b200 import binding as M
+from paper_2604_05417_b200 import build as B
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    B.build()
+    return M.load_library()
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "metasd.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(metasd_[a-z_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = declared_functions()
+    assert set(names) == set(M.EXPORTS)
+    for n in names:
+        assert getattr(lib, n) is not None
+
+
+def test_struct_mirrors_match_the_header(lib):
+    cfg = M.default_config()
+    assert C.sizeof(M.MetasdConfig) == 12 * 4 + 3 * 8
+    assert C.sizeof(M.MetasdDiag) == 20
+    assert (cfg.bandit, cfg.reward, cfg.logit_dtype, cfg.path) == (M.UCB, M.REWARD_BD, M.BF16, M.PATH_AUTO)
+    assert (cfg.beta, cfg.gamma, cfg.window, cfg.reward_temperature) == (0.01, 0.975, 50, 1.0)
+
+
+def test_host_side_validation(lib):
+    ctx = C.c_void_p()
+    bad = []
+    for field, value in [("max_batch", 0), ("max_batch", 70000), ("n_drafters", 0), ("n_drafters", 17),
+                         ("max_draft", 0), ("max_draft", 17), ("vocab", 0), ("window", 0), ("device", -1),
+                         ("beta", -1.0), ("gamma", 0.0), ("gamma", 1.5), ("reward_temperature", 0.0)]:
+        cfg = M.default_config()
+        setattr(cfg, field, value)
+        bad.append((field, lib.metasd_init(C.byref(ctx), C.byref(cfg))))
+        assert ctx.value is None
+    assert all(code == M.ERR_INVALID_ARGUMENT for _, code in bad), bad
+    for field, value in [("logit_dtype", 7), ("bandit", 3), ("reward", 2), ("path", 9)]:
+        cfg = M.default_config()
+        setattr(cfg, field, value)
+        assert lib.metasd_init(C.byref(ctx), C.byref(cfg)) == M.ERR_UNSUPPORTED
+    assert lib.metasd_init(None, C.byref(M.default_config())) == M.ERR_INVALID_ARGUMENT
+    assert lib.metasd_init(C.byref(ctx), None) == M.ERR_INVALID_ARGUMENT
+    # NULL contexts are refused everywhere
+    assert lib.metasd_select(None, 1, None, None) == M.ERR_INVALID_ARGUMENT
+    assert lib.metasd_reset(None, None, 0, None) == M.ERR_INVALID_ARGUMENT
+    assert lib.metasd_state_bytes(None) == 0
+    assert lib.metasd_kernel_launches(None) == 0
+    lib.metasd_destroy(None)
+    assert M.strerror(M.ERR_CUDA).startswith("CUDA error")
+    assert M.strerror(-99) == "unknown error"
+
+
+@pytest.mark.skipif(torch.cuda.is_available(), reason="checks the no-GPU failure mode")
+def test_no_device_is_a_loud_failure_not_a_fallback(lib):
+    with pytest.raises(M.MetasdError) as e:
+        M.MetaSD(4, 2, 3, 1000)
+    assert e.value.code == M.ERR_CUDA
+
+
+def test_missing_library_is_a_loud_failure(tmp_path):
+    with pytest.raises(FileNotFoundError):
+        M.load_library(str(tmp_path / "libmetasd.so"))
+
+
+def test_product_code_never_touches_the_oracle():
+    """The package, the header and the benchmark's own arm must not import or link oracle/."""
+    pkg = os.path.join(ROOT, "paper_2604_05417_b200")
+    for base, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                text = open(os.path.join(base, f)).read()
+                assert "oracle" not in text.lower() or f == "workloads.py", f
+    text = open(os.path.join(pkg, "workloads.py")).read()
+    assert "import oracle" not in text and "from oracle" not in text

@@ -1,0 +1,292 @@
+"""GPU parity: the CUDA library against the float64 CPU oracle on the same seeded bytes (C ABI calls)."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2604_05417_b200 import binding as M
+from paper_2604_05417_b200.workloads import WORKLOADS, RoundGenerator, Workload
+
+pytestmark = pytest.mark.gpu
+
+
+def small(name, **kw):
+    return WORKLOADS[name].scaled(**kw)
+
+
+def base(**kw):
+    d = dict(name="t", B=3, N=3, k=4, V=1000, rounds=8, temperature=1.0, dtype="bf16", bandit="ucb",
+             sigmas=(0.5, 1.5, 3.0))
+    d.update(kw)
+    return Workload(**d)
+
+
+def report(counts):
+    print({k: v for k, v in counts.items()})
+    return counts
+
+
+PATHS = [M.PATH_STREAMING, M.PATH_AUTO]
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("dtype", ["bf16", "fp32"])
+@pytest.mark.parametrize("V,k,B", [(5, 1, 1), (17, 3, 2), (1000, 4, 3), (20008, 5, 4), (4100, 16, 2), (32000, 2, 7)])
+def test_small_shapes_sampled(path, dtype, V, k, B):
+    """Tiny to several-tile vocabularies, ragged tails, scalar (V % 8 != 0) and vector rows."""
+    from _harness import run_lockstep
+    wl = base(B=B, k=k, V=V, dtype=dtype, temperature=0.8)
+    c = report(run_lockstep(wl, rounds=8, path=path))
+    assert c["rounds"] == 8
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("dtype", ["bf16", "fp32"])
+@pytest.mark.parametrize("V,k,B", [(17, 3, 2), (1000, 4, 3), (20008, 5, 4)])
+def test_small_shapes_greedy_bit_exact(path, dtype, V, k, B):
+    from _harness import run_lockstep
+    wl = base(B=B, k=k, V=V, dtype=dtype, temperature=0.0, sigmas=(0.1, 0.5, 2.0))
+    c = report(run_lockstep(wl, rounds=8, path=path))
+    assert c.get("near_tie_accept", 0) == 0 and c.get("near_tie_token", 0) == 0 and c.get("near_tie_arm", 0) == 0
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_cfg1_tiny_full_length(path):
+    from _harness import run_lockstep
+    wl = WORKLOADS["cfg1_tiny"]
+    c = report(run_lockstep(wl, rounds=wl.rounds, path=path))
+    assert c["rounds"] == 200 and c.get("near_tie_arm", 0) == 0
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("bandit", ["ducb", "swucb"])
+def test_cfg2_nonstationary_scaled(path, bandit):
+    """D-UCB and SW-UCB on the re-permuted drafter noise (period shortened so the best arm moves)."""
+    from _harness import run_lockstep
+    wl = small("cfg2_nonstationary", B=16, rounds=60, period=20, tau=15, gamma=0.9)
+    c = report(run_lockstep(wl, rounds=60, path=path, bandit=bandit))
+    assert c.get("near_tie_arm", 0) == 0
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_cfg3_tasks_scaled(path):
+    from _harness import run_lockstep
+    wl = small("cfg3_tasks", B=8, rounds=12)
+    report(run_lockstep(wl, rounds=12, path=path))
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_cfg4_greedy_scaled_bit_exact(path):
+    from _harness import run_lockstep
+    wl = small("cfg4_greedy", B=16, rounds=8)
+    c = report(run_lockstep(wl, rounds=8, path=path))
+    assert c.get("near_tie_accept", 0) == 0 and c.get("near_tie_token", 0) == 0 and c.get("near_tie_arm", 0) == 0
+
+
+@pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("bandit", ["ucb", "ducb"])
+def test_cfg5_fp32_scaled(path, bandit):
+    from _harness import run_lockstep
+    wl = small("cfg5_fp32_stress", B=8, rounds=12)
+    report(run_lockstep(wl, rounds=12, path=path, bandit=bandit))
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_pointer_table_mode(path):
+    """The kernel indexes a table of K drafter tensors and a [K,B,k] token table by arm."""
+    from _harness import run_lockstep
+    wl = base(B=5, N=4, k=3, V=4096, sigmas=(0.3, 1.0, 2.0, 3.0))
+    report(run_lockstep(wl, rounds=10, path=path, table_mode=True))
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_be_reward_mode(path):
+    from _harness import run_lockstep
+    wl = base(B=6, N=3, k=5, V=2048)
+    report(run_lockstep(wl, rounds=12, path=path, reward=M.REWARD_BE))
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_batch_shard_uses_global_sequence_ids(path):
+    """Two shards with sequence_base 0 and B/2 reproduce the unsharded results (no collective needed)."""
+    wl = base(B=8, N=2, k=3, V=1024, sigmas=(0.5, 2.0))
+    dev = torch.device("cuda", 0)
+    gen = RoundGenerator(wl, device=dev, seed=3)
+    full = M.MetaSD(8, 2, 3, 1024, path=path)
+    lo = M.MetaSD(4, 2, 3, 1024, path=path, sequence_base=0)
+    hi = M.MetaSD(4, 2, 3, 1024, path=path, sequence_base=4)
+    for t in range(5):
+        arm = full.select().cpu().numpy()
+        rd = gen.gathered_round(t, arm)
+        r = full.verify(rd["target"], rd["draft"], rd["tokens"], 1.0, 77)
+        r0 = lo.verify(rd["target"][:4].contiguous(), rd["draft"][:4].contiguous(), rd["tokens"][:4].contiguous(), 1.0, 77)
+        r1 = hi.verify(rd["target"][4:].contiguous(), rd["draft"][4:].contiguous(), rd["tokens"][4:].contiguous(), 1.0, 77)
+        for name in ("accepted_len", "next_token", "reward"):
+            assert torch.equal(getattr(r, name), torch.cat([getattr(r0, name), getattr(r1, name)]))
+        assert torch.equal(full.select(), torch.cat([lo.select(), hi.select()]))
+    for m in (full, lo, hi):
+        m.close()
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_defined_outcomes_of_anomalous_inputs(path):
+    """NaN rows, masked (-inf) logits, out-of-range tokens: same defined outputs and status bits."""
+    from _harness import make_pair, compare_round
+    wl = base(B=4, N=1, k=3, V=1024, sigmas=(1.0,))
+    dev = torch.device("cuda", 0)
+    gen = RoundGenerator(wl, device=dev, seed=5)
+    gpu, orc = make_pair(wl, path=path)
+    rd = gen.gathered_round(0, np.zeros(4, dtype=np.int64))
+    target, draft, tokens = rd["target"], rd["draft"], rd["tokens"].clone()
+    draft[0, 1, 100] = float("nan")            # sequence 0: NaN in draft row 1
+    target[1, :, 200:700] = float("-inf")      # sequence 1: masked target tokens
+    draft[1, :, 300:800] = float("-inf")
+    tokens[2, 0] = 5000                         # sequence 2: token out of range
+    tokens[3, 2] = -7
+    res = gpu.verify(target, draft, tokens, 1.0, 9, want_diag=True)
+    out = orc.verify(target, draft, tokens.cpu().numpy(), 1.0, 9)
+    compare_round(res, out, target, draft, 1.0, 1.0, {})
+    status = gpu.last_status()
+    assert status & M.STATUS_NONFINITE and status & M.STATUS_TOKEN_OOR
+    assert out["status"][0] & M.STATUS_NONFINITE and out["status"][2] & M.STATUS_TOKEN_OOR
+    assert gpu.last_status() == 0              # reading clears the word
+    gpu.close()
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_identical_drafter_accepts_everything(path):
+    wl = base(B=3, N=1, k=4, V=2048, sigmas=(0.0,))
+    dev = torch.device("cuda", 0)
+    gen = RoundGenerator(wl, device=dev, seed=6)
+    gpu = M.MetaSD(3, 1, 4, 2048, path=path)
+    rd = gen.gathered_round(0, np.zeros(3, dtype=np.int64))
+    res = gpu.verify(rd["target"], rd["target"][:, :4].contiguous(), rd["tokens"], 1.0, 1)
+    assert (res.accepted_len == 4).all()
+    assert torch.allclose(res.reward, torch.ones(3, device=dev), atol=1e-6)
+    gpu.close()
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_reset_and_state_roundtrip(path):
+    """Export -> destroy -> init -> import continues identically; reset re-initialises chosen sequences."""
+    wl = base(B=6, N=3, k=2, V=1024)
+    dev = torch.device("cuda", 0)
+    gen = RoundGenerator(wl, device=dev, seed=8)
+    a = M.MetaSD(6, 3, 2, 1024, path=path, bandit="swucb", window=4)
+    rounds = [gen.gathered_round(t, np.zeros(6, dtype=np.int64)) for t in range(8)]
+    for t in range(5):
+        a.verify(rounds[t]["target"], rounds[t]["draft"], rounds[t]["tokens"], 1.0, 3)
+    blob = a.state_export()
+    b = M.MetaSD(6, 3, 2, 1024, path=path, bandit="swucb", window=4)
+    b.state_import(blob)
+    for t in range(5, 8):
+        ra = a.verify(rounds[t]["target"], rounds[t]["draft"], rounds[t]["tokens"], 1.0, 3)
+        rb = b.verify(rounds[t]["target"], rounds[t]["draft"], rounds[t]["tokens"], 1.0, 3)
+        assert torch.equal(ra.next_token, rb.next_token) and torch.equal(ra.reward, rb.reward)
+        assert torch.equal(a.select(), b.select())
+    assert a.state_export() == b.state_export()
+    # a blob from a differently shaped context is refused
+    c = M.MetaSD(6, 3, 2, 1024, path=path, bandit="ucb", window=4)
+    with pytest.raises(M.MetasdError) as e:
+        c.state_import(blob)
+    assert e.value.code == M.ERR_BAD_STATE_BLOB
+    with pytest.raises(M.MetasdError) as e:
+        c.state_import(blob[:-8])                      # too short for this context
+    assert e.value.code == M.ERR_INVALID_ARGUMENT
+    # reset two sequences
+    a.reset(torch.tensor([1, 4], dtype=torch.int32, device=dev))
+    st = M.parse_state(a.state_export(), 6, 3, 4)
+    assert st["t"].tolist() == [8, 0, 8, 8, 0, 8] and (st["arm"][[1, 4]] == 0).all()
+    assert (st["win_reward"][[1, 4]] == 0).all()
+    a.reset()
+    assert (M.parse_state(a.state_export(), 6, 3, 4)["t"] == 0).all()
+    for m in (a, b, c):
+        m.close()
+
+
+def test_argument_validation_on_device():
+    gpu = M.MetaSD(2, 2, 3, 512)
+    dev = torch.device("cuda", 0)
+    tgt = torch.zeros((2, 4, 512), dtype=torch.bfloat16, device=dev)
+    drf = torch.zeros((2, 3, 512), dtype=torch.bfloat16, device=dev)
+    tok = torch.zeros((2, 3), dtype=torch.int32, device=dev)
+    lib, ctx = gpu.lib, gpu._ctx
+    out = [torch.zeros(2, dtype=torch.int32, device=dev), torch.zeros(2, dtype=torch.int32, device=dev),
+           torch.zeros(2, dtype=torch.float32, device=dev)]
+    import ctypes as C
+    def call(batch=2, k=3, t=tgt, d=drf, tab=None, T=1.0):
+        return lib.metasd_verify(ctx, batch, k, M._ptr(t), M._ptr(d), M._ptr(tab), M._ptr(tok), 0, C.c_float(T),
+                                 C.c_uint64(0), M._ptr(out[0]), M._ptr(out[1]), M._ptr(out[2]), None, None)
+    assert call() == M.OK
+    assert call(batch=3) == M.ERR_INVALID_ARGUMENT
+    assert call(k=4) == M.ERR_INVALID_ARGUMENT
+    assert call(k=0) == M.ERR_INVALID_ARGUMENT
+    assert call(t=None) == M.ERR_INVALID_ARGUMENT
+    assert call(d=None) == M.ERR_INVALID_ARGUMENT                       # neither draft source
+    assert call(tab=torch.zeros(2, dtype=torch.int64, device=dev)) == M.ERR_INVALID_ARGUMENT   # both
+    assert call(T=-1.0) == M.ERR_INVALID_ARGUMENT
+    assert call(T=float("nan")) == M.ERR_INVALID_ARGUMENT
+    assert lib.metasd_select(ctx, 5, M._ptr(out[0]), None) == M.ERR_INVALID_ARGUMENT
+    assert lib.metasd_verify_host(ctx, 2, 3, None, None, None, C.c_float(1.0), C.c_uint64(0), None, None, None, None,
+                                  None) == M.ERR_INVALID_ARGUMENT       # no staging in this context
+    torch.cuda.synchronize()
+    gpu.close()
+
+
+def test_verify_host_matches_device_call():
+    wl = base(B=4, N=2, k=3, V=2048, sigmas=(0.5, 2.0))
+    dev = torch.device("cuda", 0)
+    gen = RoundGenerator(wl, device=dev, seed=11)
+    a = M.MetaSD(4, 2, 3, 2048)
+    b = M.MetaSD(4, 2, 3, 2048, host_staging=True)
+    for t in range(4):
+        arm = a.select().cpu().numpy()
+        rd = gen.gathered_round(t, arm)
+        ra = a.verify(rd["target"], rd["draft"], rd["tokens"], 0.9, 21)
+        h = [x.cpu().pin_memory() for x in (rd["target"], rd["draft"], rd["tokens"])]
+        acc = torch.zeros(4, dtype=torch.int32).pin_memory()
+        tok = torch.zeros(4, dtype=torch.int32).pin_memory()
+        rew = torch.zeros(4, dtype=torch.float32).pin_memory()
+        nxt = torch.zeros(4, dtype=torch.int32).pin_memory()
+        b.verify_host(h[0], h[1], h[2], 0.9, 21, acc, tok, rew, nxt)
+        assert torch.equal(ra.accepted_len.cpu(), acc) and torch.equal(ra.next_token.cpu(), tok)
+        assert torch.equal(ra.reward.cpu(), rew) and torch.equal(a.select().cpu(), nxt)
+    a.close(); b.close()
+
+
+@pytest.mark.parametrize("name", ["cfg4_greedy", "cfg3_tasks"])
+def test_full_size_launch_sampled_against_oracle(name):
+    """The benchmark's launch configuration at full batch and vocabulary; the oracle re-computes a
+    sample of sequences one by one (each keyed by its global sequence id)."""
+    from oracle import oracle as O
+    wl = WORKLOADS[name]
+    dev = torch.device("cuda", 0)
+    gen = RoundGenerator(wl, device=dev, seed=1)
+    gpu = M.MetaSD(wl.B, wl.N, wl.k, wl.V, dtype=wl.dtype, bandit=wl.bandit)
+    sample = [0, 1, wl.B // 2 + 3, wl.B - 1]
+    T = wl.temperature
+    for t in range(2):
+        arm = gpu.select().cpu().numpy()
+        assert (arm == t).all()                       # initial sweep
+        rd = gen.gathered_round(t, arm)
+        res = gpu.verify(rd["target"], rd["draft"], rd["tokens"], T, 555, want_diag=True)
+        p_x, q_x, D, u, acc = [x.cpu().numpy() for x in res.diag_fields()]
+        n_acc = res.accepted_len.cpu().numpy()
+        assert (n_acc >= 0).all() and (n_acc <= wl.k).all()
+        rew = res.reward.cpu().numpy()
+        assert ((rew > 0) & (rew <= 1 + 1e-6)).all()
+        np.testing.assert_allclose(rew, 1 - D.mean(axis=1), atol=2e-6)
+        lead = np.where(acc.all(axis=1), wl.k, np.argmin(acc, axis=1))
+        assert np.array_equal(lead, n_acc)
+        for b in sample:
+            orc = O.OracleMetaSD(O.OracleConfig(max_batch=1, n_drafters=wl.N, vocab=wl.V, sequence_base=b))
+            orc.t[0] = t
+            out = orc.verify(rd["target"][b:b + 1], rd["draft"][b:b + 1], rd["tokens"][b:b + 1].cpu().numpy(), T, 555,
+                             update=False)
+            np.testing.assert_allclose(D[b], out["D"][0], atol=1e-5)
+            np.testing.assert_allclose(p_x[b], out["p_x"][0], atol=1e-5)
+            np.testing.assert_allclose(rew[b], out["reward"][0], atol=1e-5)
+            if T == 0 or (np.abs(out["u_accept"][0] - out["p_x"][0] / np.maximum(out["q_x"][0], 1e-300)) > 1e-6).all():
+                assert n_acc[b] == out["accepted_len"][0]
+                if T == 0 or out["sample_margin"][0] > 1e-6:
+                    assert res.next_token[b].item() == out["next_token"][0]
+    gpu.close()
