@@ -169,6 +169,39 @@ uint64_t metasd_kernel_launches(const metasd_ctx *ctx);
  * (METASD_PATH_STREAMING or METASD_PATH_FUSED). */
 int metasd_resolved_path(const metasd_ctx *ctx, int32_t k);
 
+/* One verification round for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a packaging of the stateless part of metasd_verify -- Algorithm 4 lines 6-12
+ * and the reward -- for hosts where cudaMalloc is not available to this code: a serving process whose
+ * memory pool already owns the whole device, a plugin that may not allocate after start-up, or a
+ * latency-critical thread that must stay clear of the allocator.  Such callers cannot create a
+ * context, so there is no bandit here and nothing persists between calls.)
+ *
+ * The scratch of the two kernels lives in a fixed array inside the library image (about 0.7 MB, held
+ * by every GPU that loads the library until the process exits), which bounds the sizes:
+ * batch <= METASD_NOALLOC_MAX_BATCH and batch * (k + 1) <= METASD_NOALLOC_MAX_ROWS; beyond that the
+ * call returns METASD_ERR_UNSUPPORTED and launches nothing.  The call makes no cudaMalloc / cudaFree
+ * and calls no allocating library routine.
+ *
+ * Runs on the calling thread's current device.  The first call on each device looks up the array's
+ * device address (a one-time runtime query): make that first call before any stream capture begins.
+ * All calls on a device share the one array and it keeps the previous call's contents; every field
+ * the kernels read is rewritten at the start of each call, so calls in stream order are independent,
+ * but two calls that overlap on the GPU (different streams, no ordering between them) race on it.
+ *
+ *   target_logits [batch, k+1, V], draft_logits [batch, k, V] (gathered), draft_tokens [batch, k]:
+ *   as for metasd_verify; logit_dtype is a metasd_dtype, reward_kind a metasd_reward;
+ *   reward_temperature is used only when temperature == 0 (greedy);
+ *   round is the counter that keys the uniforms with (sequence_base + b, round, position);
+ *   status_out: optional device uint32 that receives this call's METASD_STATUS_* bits. */
+#define METASD_NOALLOC_MAX_BATCH 4096
+#define METASD_NOALLOC_MAX_ROWS 16384
+int metasd_verify_noalloc(int32_t batch, int32_t k, int32_t vocab, int32_t logit_dtype,
+                          const void *target_logits, const void *draft_logits,
+                          const int32_t *draft_tokens, float temperature, float reward_temperature,
+                          int32_t reward_kind, uint64_t seed, uint32_t sequence_base, uint32_t round,
+                          int32_t *accepted_len, int32_t *next_token, float *reward,
+                          uint32_t *status_out, void *stream);
+
 const char *metasd_strerror(int code);
 
 #ifdef __cplusplus

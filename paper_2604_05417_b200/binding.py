@@ -31,7 +31,7 @@ EXPORTS = (
     "metasd_default_config", "metasd_init", "metasd_destroy", "metasd_reset", "metasd_select",
     "metasd_verify", "metasd_verify_host", "metasd_state_bytes", "metasd_state_export",
     "metasd_state_import", "metasd_last_status", "metasd_kernel_launches", "metasd_resolved_path",
-    "metasd_strerror",
+    "metasd_strerror", "metasd_verify_noalloc",
 )
 
 
@@ -90,6 +90,8 @@ def load_library(path: Optional[str] = None):
     lib.metasd_kernel_launches.argtypes = [vp]
     lib.metasd_kernel_launches.restype = u64
     lib.metasd_resolved_path.argtypes = [vp, i32]
+    lib.metasd_verify_noalloc.argtypes = [i32, i32, i32, i32, vp, vp, vp, C.c_float, C.c_float, i32, u64, C.c_uint32,
+                                          C.c_uint32, vp, vp, vp, vp, vp]
     lib.metasd_strerror.argtypes = [C.c_int]
     lib.metasd_strerror.restype = C.c_char_p
     if path == LIB_PATH:
@@ -232,6 +234,21 @@ class MetaSD:
 
     def resolved_path(self, k: int) -> int:
         return int(self.lib.metasd_resolved_path(self._ctx, k))
+
+
+def verify_noalloc(target_logits: torch.Tensor, draft_logits: torch.Tensor, draft_tokens: torch.Tensor,
+                   temperature: float, seed: int, round_: int, accepted_len: torch.Tensor,
+                   next_token: torch.Tensor, reward: torch.Tensor, status: Optional[torch.Tensor] = None,
+                   sequence_base: int = 0, reward_temperature: float = 1.0, reward_kind: int = REWARD_BD) -> int:
+    """metasd_verify_noalloc on the current device and stream: no context, no allocation inside the
+    library; the caller provides every buffer.  Returns the library's error code."""
+    B, kp1, V = target_logits.shape
+    dev = target_logits.device
+    return load_library().metasd_verify_noalloc(
+        B, kp1 - 1, V, DTYPES[target_logits.dtype], _ptr(target_logits), _ptr(draft_logits), _ptr(draft_tokens),
+        C.c_float(temperature), C.c_float(reward_temperature), reward_kind, C.c_uint64(seed),
+        C.c_uint32(sequence_base), C.c_uint32(round_), _ptr(accepted_len), _ptr(next_token), _ptr(reward),
+        _ptr(status), _stream(dev))
 
 
 def pointer_table(tensors: Sequence[torch.Tensor]) -> torch.Tensor:
