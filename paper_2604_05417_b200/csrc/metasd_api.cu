@@ -21,6 +21,7 @@ struct metasd_ctx {
     int32_t *stage_tokens, *stage_acc, *stage_tok;
     float *stage_reward;
     bool fused_ready;
+    FusedPlan plan;
 };
 
 namespace {
@@ -136,7 +137,7 @@ int metasd_init(metasd_ctx **out, const metasd_config *cfg)
     if (e == cudaSuccess) e = launch_reset(c->st, cfg->max_batch, cfg->n_drafters, cfg->window, nullptr, cfg->max_batch, 0);
     if (e == cudaSuccess && cfg->path != METASD_PATH_STREAMING &&
         fused_supported(cfg->logit_dtype, cfg->vocab, cfg->max_draft)) {
-        e = fused_prepare(cfg->device);
+        e = fused_prepare(cfg->device, cfg->logit_dtype, cfg->vocab, cfg->max_batch, &c->plan);
         c->fused_ready = (e == cudaSuccess);
         if (cfg->path == METASD_PATH_AUTO && e != cudaSuccess) { (void)cudaGetLastError(); e = cudaSuccess; }
     }
@@ -216,7 +217,7 @@ int metasd_verify(metasd_ctx *ctx, int32_t batch, int32_t k, const void *target_
 
     cudaError_t e;
     if (metasd_resolved_path(ctx, k) == METASD_PATH_FUSED && p.vector_ok)
-        e = launch_fused(p, cfg.logit_dtype, (cudaStream_t)stream, &ctx->launches);
+        e = launch_fused(p, cfg.logit_dtype, ctx->plan, (cudaStream_t)stream, &ctx->launches);
     else if (cfg.path == METASD_PATH_FUSED)
         return METASD_ERR_UNSUPPORTED;
     else

@@ -59,9 +59,21 @@ struct VerifyParams {
 // streaming path (metasd_streaming.cu)
 cudaError_t launch_streaming(const VerifyParams &p, int dtype, cudaStream_t stream, uint64_t *launches);
 // fused cluster path (metasd_fused.cu)
+struct FusedPlan {
+    int32_t cluster;       // CTAs per cluster (0: no plan)
+    int32_t threads;       // threads per CTA
+    int32_t n_vec_row;     // 16-byte vectors per logit row
+    int32_t n_vec_cta;     // vectors of a row owned by one CTA
+    int32_t n_slot;        // ring slots of slot_bytes each
+    int32_t slot_bytes;
+    int32_t max_clusters;  // co-resident clusters on the device
+    size_t smem_bytes;     // dynamic shared memory of the launch
+    long work_per_item;    // threads x vectors per thread
+};
 bool fused_supported(int dtype, int V, int k);
-cudaError_t fused_prepare(int device);
-cudaError_t launch_fused(const VerifyParams &p, int dtype, cudaStream_t stream, uint64_t *launches);
+cudaError_t fused_prepare(int device, int dtype, int V, int max_batch, FusedPlan *plan);
+cudaError_t launch_fused(const VerifyParams &p, int dtype, const FusedPlan &plan, cudaStream_t stream,
+                         uint64_t *launches);
 // small state kernels (metasd_streaming.cu)
 cudaError_t launch_select(const BanditState &st, int batch, int32_t *arm_out, cudaStream_t stream);
 cudaError_t launch_reset(const BanditState &st, int max_batch, int K, int tau, const int32_t *seq_ids,
