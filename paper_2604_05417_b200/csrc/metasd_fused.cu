@@ -75,10 +75,6 @@ __device__ __forceinline__ uint32_t map_to_rank(uint32_t local, uint32_t rank)
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local), "r"(rank));
     return r;
 }
-__device__ __forceinline__ void st_cluster(uint32_t addr, float v)
-{
-    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
-}
 __device__ __forceinline__ void st_cluster(uint32_t addr, int32_t v)
 {
     asm volatile("st.shared::cluster.s32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
@@ -127,31 +123,41 @@ __device__ __forceinline__ float warp_sum_f(float v)
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
     return v;
 }
+// Warp-wide maximum in one instruction (sm_100a).
 __device__ __forceinline__ float warp_max_f(float v)
 {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
-    return v;
+    float r;
+    asm volatile("redux.sync.max.f32 %0, %1, 0xffffffff;" : "=f"(r) : "f"(v));
+    return r;
+}
+// 16 bytes into a peer CTA's shared memory; the peer's mbarrier counts them as transferred bytes.
+__device__ __forceinline__ void st_async_16(uint32_t remote_addr, uint32_t remote_bar, uint32_t a, uint32_t b, uint32_t c,
+                                            uint32_t d)
+{
+    asm volatile("st.async.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];"
+                 ::"r"(remote_addr), "r"(a), "r"(b), "r"(c), "r"(d), "r"(remote_bar)
+                 : "memory");
 }
 
 // ---------------------------------------------------------------------------------------------
 // Shared-memory state of one CTA (besides the ring)
 // ---------------------------------------------------------------------------------------------
-struct __align__(16) Exchange {   // what one CTA tells the cluster about its slice of a row pair
+struct __align__(16) Exchange {   // (max, sum) of both rows and the first arg-max of the target row
     float max_a, sum_a, max_b, sum_b;
-    int32_t idx_a;                // first index of max_a inside the slice
+    int32_t idx_a;
     int32_t pad[3];
 };
+constexpr uint32_t EXCHANGE_BYTES = 32;
 
 struct FusedShared {
     uint64_t full[FUSED_MAX_SLOTS];                      // one mbarrier per ring slot
+    uint64_t xbar[2];                                    // arrival of the peers' records, by item parity
     Exchange exch[2][FUSED_MAX_CLUSTER];                 // [item parity][sender rank]
+    Exchange wrec[2][FUSED_MAX_WARPS];                   // [item parity][warp]: the warps' records
     double tot[10 * FUSED_MAX_WARPS];                    // draw: weight of (vector index i, warp)
     double pre[10 * FUSED_MAX_WARPS];                    // draw: exclusive prefix of tot
     double cta_tot[FUSED_MAX_CLUSTER];                   // draw: weight of each CTA's slice
     double cta_min[16][FUSED_MAX_CLUSTER];               // rank 0: sum of min(p, q) per position and sender
-    float wmax[2][FUSED_MAX_WARPS];
-    float wsum[2][FUSED_MAX_WARPS];
     float pmin[16][FUSED_MAX_WARPS];                     // sum of min(p, q) per position and warp
     const void *table[16];                               // the drafter pointer table
     // header of the current sequence
@@ -162,7 +168,6 @@ struct FusedShared {
     int32_t r_acc[16];
     float r_px[16], r_qx[16];
     uint32_t r_rowflag[16];
-    int32_t idx;        // arg-max candidate of this CTA's slice
     int32_t nstar, nlast, token;
     int32_t dead;       // a wait ran out: later waits do not spin again
 };
@@ -174,11 +179,11 @@ struct FusedGeom {
     int32_t slot_bytes;  // n_vec_cta * 16
 };
 
-// Waits for a ring slot.  Bounded: after the limit the CTA is marked dead, the status word gets the
-// time-out bit and every later wait returns at once, so all barriers stay matched and the kernel ends.
-__device__ __forceinline__ void wait_slot(FusedShared &sh, int slot, uint32_t parity, uint32_t *status)
+// Waits for a phase of an mbarrier.  Bounded: after the limit the CTA is marked dead, the status word
+// gets the time-out bit and every later wait returns at once, so all barriers stay matched, every CTA
+// still sends its records and the kernel ends.
+__device__ __forceinline__ void wait_bar(FusedShared &sh, uint64_t *bar, uint32_t parity, uint32_t *status)
 {
-    uint64_t *bar = &sh.full[slot];
     if (mbar_try_wait(bar, parity)) return;
     if (*(volatile int32_t *)&sh.dead) return;
     for (uint32_t it = 0; it < WAIT_FAST_POLLS + WAIT_SLOW_POLLS; ++it) {
@@ -189,38 +194,103 @@ __device__ __forceinline__ void wait_slot(FusedShared &sh, int slot, uint32_t pa
     atomicOr(status, METASD_STATUS_TIMEOUT);
 }
 
-// One row slice from shared memory into registers: e[q] = 2^((x_q - m_t) c) with the thread's own
-// maximum m_t, s_t = sum_q e[q].  Vector i of the thread is vector i * nthr + tid of the slice.
+// Element q of a register array of pairs.
+template <int N>
+__device__ __forceinline__ float elem(const float2 (&a)[N], int q) { return (q & 1) ? a[q >> 1].y : a[q >> 1].x; }
+
+// One row slice from shared memory into registers: e_q = 2^((x_q - m_t) c) with the thread's own
+// maximum m_t, s_t = sum_q e_q.  Vector i of the thread is vector i * nthr + tid of the slice.
 template <typename LT, int VPT>
 __device__ __forceinline__ void load_row(const unsigned char *slot, int my_vecs, int tid, int nthr, float c,
-                                         float (&e)[VPT * Logit<LT>::VEC], float &m_t, float &s_t)
+                                         float2 (&e)[VPT * Logit<LT>::VEC / 2], float &m_t, float &s_t)
 {
-    constexpr int VEC = Logit<LT>::VEC;
-    // every lane of a vector outside the slice reads as -inf: weight 0, never the maximum
-    const uint32_t ninf = sizeof(LT) == 2 ? 0xFF80FF80u : 0xFF800000u;
+    constexpr int NP = VPT * Logit<LT>::VEC / 2;
     float m = METASD_NEG_BIG;
+    if constexpr (sizeof(LT) == 2) {
+        // every lane of a vector outside the slice reads as -inf: weight 0, never the maximum
+        uint32_t w[NP];
 #pragma unroll
-    for (int i = 0; i < VPT; ++i) {
-        const int v = i * nthr + tid;
-        uint4 raw = make_uint4(ninf, ninf, ninf, ninf);
-        if (v < my_vecs) raw = *reinterpret_cast<const uint4 *>(slot + (size_t)v * 16);
-        float x[VEC];
-        Logit<LT>::unpack(raw, x);
+        for (int i = 0; i < VPT; ++i) {
+            const int v = i * nthr + tid;
+            uint4 raw = make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);
+            if (v < my_vecs) raw = *reinterpret_cast<const uint4 *>(slot + (size_t)v * 16);
+            w[4 * i] = raw.x; w[4 * i + 1] = raw.y; w[4 * i + 2] = raw.z; w[4 * i + 3] = raw.w;
+        }
+        // the maximum on the packed words, two logits per instruction
+        __nv_bfloat162 m2 = *reinterpret_cast<const __nv_bfloat162 *>(&w[0]);
 #pragma unroll
-        for (int q = 0; q < VEC; ++q) {
-            e[i * VEC + q] = x[q];
-            m = fmaxf(m, x[q]);
+        for (int n = 1; n < NP; ++n) m2 = __hmax2(m2, *reinterpret_cast<const __nv_bfloat162 *>(&w[n]));
+        m = fmaxf(m, fmaxf(__low2float(m2), __high2float(m2)));
+#pragma unroll
+        for (int n = 0; n < NP; ++n) e[n] = make_float2(__uint_as_float(w[n] << 16), __uint_as_float(w[n] & 0xFFFF0000u));
+    } else {
+#pragma unroll
+        for (int i = 0; i < VPT; ++i) {
+            const int v = i * nthr + tid;
+            uint4 raw = make_uint4(0xFF800000u, 0xFF800000u, 0xFF800000u, 0xFF800000u);
+            if (v < my_vecs) raw = *reinterpret_cast<const uint4 *>(slot + (size_t)v * 16);
+            e[2 * i] = make_float2(__uint_as_float(raw.x), __uint_as_float(raw.y));
+            e[2 * i + 1] = make_float2(__uint_as_float(raw.z), __uint_as_float(raw.w));
+            m = fmaxf(m, fmaxf(fmaxf(e[2 * i].x, e[2 * i].y), fmaxf(e[2 * i + 1].x, e[2 * i + 1].y)));
         }
     }
     const float nm = -m * c;
-    float s = 0.f;
+    const float2 cc = make_float2(c, c), nn = make_float2(nm, nm);
+    float2 s2 = make_float2(0.f, 0.f);
 #pragma unroll
-    for (int q = 0; q < VPT * VEC; ++q) {
-        e[q] = ex2(fmaf(e[q], c, nm));
-        s += e[q];
+    for (int n = 0; n < NP; ++n) {
+        const float2 y = __ffma2_rn(e[n], cc, nn);
+        e[n] = make_float2(ex2(y.x), ex2(y.y));
+        s2 = __fadd2_rn(s2, e[n]);
     }
     m_t = m;
-    s_t = s;
+    s_t = s2.x + s2.y;
+}
+
+// First index (in the row) of value m among this thread's logits of a slice, INT_MAX if absent.
+template <typename LT, int VPT>
+__device__ __forceinline__ int first_index_of(const unsigned char *slot, int my_vecs, int tid, int nthr, int vec0, float m)
+{
+    constexpr int VEC = Logit<LT>::VEC;
+    int found = INT_MAX;
+#pragma unroll
+    for (int i = VPT - 1; i >= 0; --i) {
+        const int v = i * nthr + tid;
+        if (v < my_vecs) {
+            float x[VEC];
+            Logit<LT>::unpack(*reinterpret_cast<const uint4 *>(slot + (size_t)v * 16), x);
+#pragma unroll
+            for (int q = VEC - 1; q >= 0; --q)
+                if (x[q] == m) found = (vec0 + v) * VEC + q;
+        }
+    }
+    return found;
+}
+
+// Merges up to 32 records held one per lane (lanes >= n hold nothing): row maxima, row sums relative
+// to them, the first arg-max of the target row, and each lane's own rescaling factors.
+struct Merged {
+    float Ma, Sa, Mb, Sb;
+    int idx;
+    float ta, tb;   // this lane's 2^((m_lane - M) c)
+};
+__device__ __forceinline__ Merged merge_records(const Exchange *rec, int n, int lane, float c)
+{
+    float ma = METASD_NEG_BIG, sa = 0.f, mb = METASD_NEG_BIG, sb = 0.f;
+    int ia = INT_MAX;
+    if (lane < n) {
+        const Exchange x = rec[lane];
+        ma = x.max_a; sa = x.sum_a; mb = x.max_b; sb = x.sum_b; ia = x.idx_a;
+    }
+    Merged r;
+    r.Ma = warp_max_f(ma);
+    r.Mb = warp_max_f(mb);
+    r.ta = ex2((ma - r.Ma) * c);
+    r.tb = ex2((mb - r.Mb) * c);
+    r.Sa = warp_sum_f(sa * r.ta);
+    r.Sb = warp_sum_f(sb * r.tb);
+    r.idx = __reduce_min_sync(0xFFFFFFFFu, (lane < n && ma == r.Ma) ? ia : INT_MAX);
+    return r;
 }
 
 // Weight of element q in the draw: mode 1 = max(0, p - q) (correction), mode 2 = p (bonus).
@@ -235,7 +305,7 @@ __device__ __forceinline__ float draw_weight(int mode, float ea, float fa, float
 // of the vector).  Totals and offsets are carried in fp64.  Returns false (for every thread of the
 // cluster alike) when the row has no mass; otherwise the token lands in sh.token of rank 0.
 template <int VPT, int VEC>
-__device__ bool cluster_draw(FusedShared &sh, const float (&ea)[VPT * VEC], const float (&eb)[VPT * VEC], float fa,
+__device__ bool cluster_draw(FusedShared &sh, const float2 (&ea)[VPT * VEC / 2], const float2 (&eb)[VPT * VEC / 2], float fa,
                              float fb, int mode, float u, int rank, int csize, int vec0, int nthr)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -245,7 +315,7 @@ __device__ bool cluster_draw(FusedShared &sh, const float (&ea)[VPT * VEC], cons
     for (int i = 0; i < VPT; ++i) {
         float s = 0.f;
 #pragma unroll
-        for (int q = 0; q < VEC; ++q) s += draw_weight(mode, ea[i * VEC + q], fa, eb[i * VEC + q], fb);
+        for (int q = 0; q < VEC; ++q) s += draw_weight(mode, elem(ea, i * VEC + q), fa, elem(eb, i * VEC + q), fb);
         vs[i] = s;
     }
     if (tid == 0) { sh.nstar = INT_MAX; sh.nlast = -1; }
@@ -335,7 +405,7 @@ __device__ bool cluster_draw(FusedShared &sh, const float (&ea)[VPT * VEC], cons
                     if (i == istar) {
 #pragma unroll
                         for (int q = 0; q < VEC; ++q) {
-                            const float w = draw_weight(mode, ea[i * VEC + q], fa, eb[i * VEC + q], fb);
+                            const float w = draw_weight(mode, elem(ea, i * VEC + q), fa, elem(eb, i * VEC + q), fb);
                             cum += (double)w;
                             if (w > 0.f) last_q = q;
                             if (tok_q < 0 && cum > th) tok_q = q;
@@ -422,7 +492,7 @@ template <typename LT, int VPT>
 __global__ void __launch_bounds__(FUSED_MAX_THREADS, 1) fused_round_kernel(const VerifyParams p, const FusedGeom g)
 {
     constexpr int VEC = Logit<LT>::VEC;
-    constexpr int EPT = VPT * VEC;
+    constexpr int NP = VPT * VEC / 2;
     extern __shared__ __align__(128) unsigned char ring[];
     __shared__ FusedShared sh;
 
@@ -439,12 +509,14 @@ __global__ void __launch_bounds__(FUSED_MAX_THREADS, 1) fused_round_kernel(const
 
     if (tid == 0) {
         for (int s = 0; s < g.n_slot; ++s) mbar_init(&sh.full[s], 1);
+        mbar_init(&sh.xbar[0], 1);
+        mbar_init(&sh.xbar[1], 1);
         sh.dead = 0;
         sh.token = -1;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (tid < 16) sh.table[tid] = (p.drafter_ptrs && tid < p.K) ? p.drafter_ptrs[tid] : nullptr;
-    cluster_sync_all();   // every CTA of the cluster is running before anyone writes into a peer's shared memory
+    cluster_sync_all();   // every CTA of the cluster is running, its barriers initialised, before a peer writes to it
 
     // ---- producer (thread 0): the order of loads is sequence-major, position, target then draft
     int ld_b = cid, ld_j = 0, ld_row = 0, ld_slot = 0, ld_arm_next = 0;
@@ -454,7 +526,7 @@ __global__ void __launch_bounds__(FUSED_MAX_THREADS, 1) fused_round_kernel(const
         return reinterpret_cast<const unsigned char *>(p.draft ? p.draft : sh.table[arm & 15]);
     };
     auto issue_one = [&]() {
-        if (ld_b >= p.batch) return;
+        if (ld_b >= p.batch || *(volatile int32_t *)&sh.dead) return;   // after a time-out nothing more is armed
         const unsigned char *base = ld_row == 0 ? reinterpret_cast<const unsigned char *>(p.target) : ld_draft;
         const unsigned char *src =
             base + (ld_row == 0 ? ((size_t)ld_b * (k + 1) + ld_j) : ((size_t)ld_b * k + ld_j)) * row_bytes + (size_t)vec0 * 16;
@@ -522,7 +594,7 @@ __global__ void __launch_bounds__(FUSED_MAX_THREADS, 1) fused_round_kernel(const
 
     int cs = 0;              // ring slot the consumers read next
     uint32_t cpar = 0;       // and its phase parity
-    uint32_t item = 0;       // items done by this cluster (parity of the exchange buffers)
+    uint32_t item = 0;       // items done by this cluster: bit 0 selects the exchange buffers, bit 1 their phase
 
     for (int b = cid; b < p.batch; b += ncl) {
         // ---- publish the header of sequence b
@@ -548,57 +620,51 @@ __global__ void __launch_bounds__(FUSED_MAX_THREADS, 1) fused_round_kernel(const
         for (int j = 0; j <= k; ++j, ++item) {
             const bool pair = j < k;
             const int par = item & 1;
-            if (warp == 0 && b_next < p.batch) {
-                if (j == 0) fetch_step(b_next, 0);
-                if (j == 1) fetch_step(b_next, 1);
-                if (j == (k < 2 ? k : 2)) fetch_step(b_next, 2);
+            if (warp == 0) {
+                if (b_next < p.batch) {
+                    if (j == 0) fetch_step(b_next, 0);
+                    if (j == 1) fetch_step(b_next, 1);
+                    if (j == (k < 2 ? k : 2)) fetch_step(b_next, 2);
+                }
+                // expect one record of 32 bytes from every CTA of the cluster (this one included)
+                if (lane == 0 && !*(volatile int32_t *)&sh.dead)
+                    mbar_arrive_expect_tx(&sh.xbar[par], (uint32_t)csize * EXCHANGE_BYTES);
             }
-            if (tid == 0) sh.idx = INT_MAX;
 
-            // ---- this item's slices: shared memory -> registers, exponentials relative to the thread maximum
-            float ea[EPT], eb[EPT];
-            float mta, sta, mtb = METASD_NEG_BIG, stb = 0.f;
-            const int slot_a = cs;
-            wait_slot(sh, cs, cpar, p.status);
-            load_row<LT, VPT>(ring + (size_t)cs * g.slot_bytes, my_vecs, tid, nthr, c, ea, mta, sta);
-            if (++cs == g.n_slot) { cs = 0; cpar ^= 1u; }
+            // ---- this item's slices: shared memory -> registers, exponentials relative to the thread maximum,
+            //      then the warp's record: maxima, sums relative to them, first arg-max of the target row
+            float2 ea[NP], eb[NP];
+            float mta, mtb = METASD_NEG_BIG;
+            Exchange wr;
+            {
+                float sta;
+                const unsigned char *slot = ring + (size_t)cs * g.slot_bytes;
+                wait_bar(sh, &sh.full[cs], cpar, p.status);
+                load_row<LT, VPT>(slot, my_vecs, tid, nthr, c, ea, mta, sta);
+                if (++cs == g.n_slot) { cs = 0; cpar ^= 1u; }
+                wr.max_a = warp_max_f(mta);
+                wr.sum_a = warp_sum_f(sta * ex2((mta - wr.max_a) * c));
+                int cand = INT_MAX;
+                if (p.greedy && mta == wr.max_a && mta > METASD_NEG_BIG)
+                    cand = first_index_of<LT, VPT>(slot, my_vecs, tid, nthr, vec0, mta);
+                wr.idx_a = p.greedy ? __reduce_min_sync(0xFFFFFFFFu, cand) : INT_MAX;
+            }
             if (pair) {
-                wait_slot(sh, cs, cpar, p.status);
+                float stb;
+                wait_bar(sh, &sh.full[cs], cpar, p.status);
                 load_row<LT, VPT>(ring + (size_t)cs * g.slot_bytes, my_vecs, tid, nthr, c, eb, mtb, stb);
                 if (++cs == g.n_slot) { cs = 0; cpar ^= 1u; }
+                wr.max_b = warp_max_f(mtb);
+                wr.sum_b = warp_sum_f(stb * ex2((mtb - wr.max_b) * c));
             } else {
 #pragma unroll
-                for (int q = 0; q < EPT; ++q) eb[q] = 0.f;
+                for (int n = 0; n < NP; ++n) eb[n] = make_float2(0.f, 0.f);
+                wr.max_b = METASD_NEG_BIG;
+                wr.sum_b = 0.f;
             }
-            {
-                const float wa_ = warp_max_f(mta), wb_ = warp_max_f(mtb);
-                if (lane == 0) { sh.wmax[0][warp] = wa_; sh.wmax[1][warp] = wb_; }
-            }
-            __syncthreads();
-
-            // ---- CTA maxima; the first index of the target maximum; sums relative to the CTA maxima
-            float cma = METASD_NEG_BIG, cmb = METASD_NEG_BIG;
-            for (int w = 0; w < nw; ++w) { cma = fmaxf(cma, sh.wmax[0][w]); cmb = fmaxf(cmb, sh.wmax[1][w]); }
-            if (mta == cma && cma > METASD_NEG_BIG) {
-                const unsigned char *slot = ring + (size_t)slot_a * g.slot_bytes;
-                int found = INT_MAX;
-#pragma unroll
-                for (int i = VPT - 1; i >= 0; --i) {
-                    const int v = i * nthr + tid;
-                    if (v < my_vecs) {
-                        float x[VEC];
-                        Logit<LT>::unpack(*reinterpret_cast<const uint4 *>(slot + (size_t)v * 16), x);
-#pragma unroll
-                        for (int q = VEC - 1; q >= 0; --q)
-                            if (x[q] == cma) found = (vec0 + v) * VEC + q;
-                    }
-                }
-                atomicMin(&sh.idx, found);
-            }
-            const float ga = ex2((mta - cma) * c), gb = ex2((mtb - cmb) * c);
-            {
-                const float wa_ = warp_sum_f(sta * ga), wb_ = warp_sum_f(stb * gb);
-                if (lane == 0) { sh.wsum[0][warp] = wa_; sh.wsum[1][warp] = wb_; }
+            if (lane == 0) {
+                wr.pad[0] = wr.pad[1] = wr.pad[2] = 0;
+                sh.wrec[par][warp] = wr;
             }
             __syncthreads();
 
@@ -609,61 +675,42 @@ __global__ void __launch_bounds__(FUSED_MAX_THREADS, 1) fused_round_kernel(const
                 issue_one();
                 if (pair) issue_one();
             }
-            // ---- tell the cluster
+            // ---- the CTA's record goes to every CTA of the cluster (asynchronous stores that complete on
+            //      the receiver's barrier); then wait for all the records addressed to this CTA
             if (warp == 0) {
-                float s_a = lane < nw ? sh.wsum[0][lane] : 0.f;
-                float s_b = lane < nw ? sh.wsum[1][lane] : 0.f;
-                s_a = warp_sum_f(s_a);
-                s_b = warp_sum_f(s_b);
+                const Merged mc = merge_records(sh.wrec[par], nw, lane, c);
                 if (lane < csize) {
                     const uint32_t dst = map_to_rank(smem_addr(&sh.exch[par][rank]), (uint32_t)lane);
-                    st_cluster(dst + 0, cma);
-                    st_cluster(dst + 4, s_a);
-                    st_cluster(dst + 8, cmb);
-                    st_cluster(dst + 12, s_b);
-                    st_cluster(dst + 16, sh.idx);
+                    const uint32_t bar = map_to_rank(smem_addr(&sh.xbar[par]), (uint32_t)lane);
+                    st_async_16(dst, bar, __float_as_uint(mc.Ma), __float_as_uint(mc.Sa), __float_as_uint(mc.Mb),
+                                __float_as_uint(mc.Sb));
+                    st_async_16(dst + 16, bar, (uint32_t)mc.idx, 0u, 0u, 0u);
                 }
             }
-            cluster_sync_all();
+            wait_bar(sh, &sh.xbar[par], (item >> 1) & 1u, p.status);
+            const Merged mg = merge_records(sh.exch[par], csize, lane, c);
+            const float Ma = mg.Ma, Sa = mg.Sa, Mb = mg.Mb, Sb = mg.Sb;
+            const int argidx = mg.idx;
 
-            // ---- merge the records (every warp alike): row maxima, row sums, arg-max, this CTA's factors
-            float Ma, Sa, Mb, Sb, ha, hb;
-            int argidx;
-            {
-                float ma = METASD_NEG_BIG, sa_ = 0.f, mb = METASD_NEG_BIG, sb_ = 0.f;
-                int ia = INT_MAX;
-                if (lane < csize) {
-                    const Exchange &x = sh.exch[par][lane];
-                    ma = x.max_a; sa_ = x.sum_a; mb = x.max_b; sb_ = x.sum_b; ia = x.idx_a;
-                }
-                Ma = warp_max_f(ma);
-                Mb = warp_max_f(mb);
-                const float ta = ex2((ma - Ma) * c), tb = ex2((mb - Mb) * c);
-                Sa = warp_sum_f(sa_ * ta);
-                Sb = warp_sum_f(sb_ * tb);
-                ha = __shfl_sync(0xFFFFFFFFu, ta, rank);
-                hb = __shfl_sync(0xFFFFFFFFu, tb, rank);
-                int cand = (lane < csize && ma == Ma) ? ia : INT_MAX;
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) cand = min(cand, __shfl_xor_sync(0xFFFFFFFFu, cand, o));
-                argidx = cand;
-            }
             // NaN or +Inf anywhere makes the sum NaN; an all -Inf row leaves it 0
             const bool bad_a = !(Sa > 0.f) || !(Sa < INFINITY) || !(Ma < INFINITY);
             const bool bad_b = pair && (!(Sb > 0.f) || !(Sb < INFINITY) || !(Mb < INFINITY));
             const uint32_t rowflag = (bad_a || bad_b) ? METASD_STATUS_NONFINITE : 0u;
-            const float fa = rowflag ? 0.f : ga * ha / Sa;
-            const float fb = (rowflag || !pair) ? 0.f : gb * hb / Sb;
+            // p_v = e_v * fa with fa = 2^((m_t - M) c) / S
+            const float fa = rowflag ? 0.f : ex2((mta - Ma) * c) / Sa;
+            const float fb = (rowflag || !pair) ? 0.f : ex2((mtb - Mb) * c) / Sb;
 
-            // ---- sum_v min(p_v, q_v) of this CTA's slice
+            // ---- sum_v min(p_v, q_v) of this warp's logits
             bool accepted = false;
             if (pair) {
-                float acc = 0.f;
-                if (!rowflag) {
+                float2 acc2 = make_float2(0.f, 0.f);
+                const float2 fa2 = make_float2(fa, fa), fb2 = make_float2(fb, fb);
 #pragma unroll
-                    for (int q = 0; q < EPT; ++q) acc += fminf(ea[q] * fa, eb[q] * fb);
+                for (int n = 0; n < NP; ++n) {
+                    const float2 pv = __fmul2_rn(ea[n], fa2), qv = __fmul2_rn(eb[n], fb2);
+                    acc2 = __fadd2_rn(acc2, make_float2(fminf(pv.x, qv.x), fminf(pv.y, qv.y)));
                 }
-                acc = warp_sum_f(acc);
+                const float acc = warp_sum_f(acc2.x + acc2.y);
                 if (lane == 0) sh.pmin[j][warp] = acc;
 
                 // ---- the accept test of Algorithm 4 (lines 7-8), evaluated alike by every thread of the cluster
@@ -758,7 +805,7 @@ __global__ void __launch_bounds__(FUSED_MAX_THREADS, 1) fused_round_kernel(const
     // ---- no CTA leaves while a copy into its shared memory may be in flight or a peer may still write to it
     if (tid == 0) {
         while (consumed < ld_issued) {
-            wait_slot(sh, cs, cpar, p.status);
+            wait_bar(sh, &sh.full[cs], cpar, p.status);
             if (++cs == g.n_slot) { cs = 0; cpar ^= 1u; }
             ++consumed;
         }
