@@ -2,18 +2,25 @@
 //
 // A thread-block cluster of C CTAs owns one sequence at a time and walks its k+1 positions in order.
 // Every CTA owns a contiguous 1/C slice of each logit row.  The slices arrive in shared memory through
-// a ring of bulk asynchronous copies (TMA, completion on an mbarrier) that runs several rows ahead of
-// the arithmetic, so each logit is read from HBM exactly once.  A thread turns its logits into
-// exponentials relative to its own maximum and keeps them in registers; the cluster exchanges
-// (max, sum, arg-max) records through distributed shared memory, after which the same registers give
-//   - sum_v min(p_v, q_v) = 1 - d_TV(p_j, q_j)                                (Definition 2, Eq. 4),
-//   - the accept test u q(x) < p(x) of the drafted token                      (Algorithm 4, lines 7-8),
-//   - at the first rejection (or at the bonus position) the inverse-CDF draw from max(0, p - q)
-//     (or from p), a prefix search in token order across the cluster          (Algorithm 4, lines 11-12).
-// Rank 0 of the cluster then writes the outputs, forms the reward and a warp updates the bandit and
-// selects the next arm with one lane per drafter                             (Algorithm 2, lines 7-10).
+// a ring of bulk asynchronous copies (TMA, completion on an mbarrier) that runs ahead of the arithmetic,
+// so each logit is read from HBM exactly once and stays on chip for both passes over it:
 //
-// One exponential is evaluated per logit (the special-function pipe is the second roof of this path).
+//   pass 1 (row statistics)  per row: running maximum and sum_v 2^((x_v - max) c); the CTA's record
+//                            (max, sum, first arg-max) goes to every CTA of the cluster as asynchronous
+//                            distributed-shared-memory stores that complete on the receiver's mbarrier;
+//   pass 2 (one item later)  with the merged records of the whole row pair:
+//                              sum_v min(p_v, q_v) = 1 - d_TV(p_j, q_j)            (Definition 2, Eq. 4)
+//                            evaluated as sum_v 2^min(log2 p_v, log2 q_v): one exponential per PAIR;
+//                            the accept test u q(x) < p(x) of the drafted token     (Algorithm 4, l. 7-8);
+//                            at the first rejection (or the bonus position) the inverse-CDF draw from
+//                            max(0, p - q) (or p), a prefix search in token order across the cluster
+//                                                                                    (Algorithm 4, l. 11-12).
+//
+// Pass 2 of item n-1 runs after pass 1 of item n, so the latency of the record exchange hides behind a
+// full pass.  Warp 0 of every CTA is a control warp (lane j = position j of the sequence): it issues the
+// copies, merges and sends records, runs the accept tests, and in rank 0 writes the outputs, forms the
+// reward and updates the bandit with one lane per drafter (Algorithm 2, lines 7-10).  The other warps
+// only stream logits out of shared memory.
 #include <limits.h>
 #include <stdio.h>
 #include <stdlib.h>
@@ -24,11 +31,11 @@ namespace metasd {
 
 namespace {
 
-constexpr int FUSED_MAX_THREADS = 512;
+constexpr int FUSED_MAX_THREADS = 1024;
 constexpr int FUSED_MAX_WARPS = FUSED_MAX_THREADS / 32;
 constexpr int FUSED_MAX_CLUSTER = 16;
 constexpr int FUSED_MAX_SLOTS = 8;
-constexpr int FUSED_MAX_POS = 17;                 // k + 1 <= 17
+constexpr int FUSED_MIN_SLOTS = 5;                // two items of two rows each, plus one copy in flight
 constexpr int FUSED_SMEM_RESERVE = 12 * 1024;     // static shared memory + slack kept out of the ring
 constexpr uint32_t WAIT_FAST_POLLS = 4096u;
 constexpr uint32_t WAIT_SLOW_POLLS = 1u << 21;    // with a back-off of 128 ns each: a few tenths of a second
@@ -149,27 +156,30 @@ struct __align__(16) Exchange {   // (max, sum) of both rows and the first arg-m
 };
 constexpr uint32_t EXCHANGE_BYTES = 32;
 
+// What the control warp hands to the streaming warps for pass 2 of one item.
+struct RowConst {
+    float nma, nmb;      // -max c of the target / draft row
+    float nmb_rel;       // nmb + log2(sum_a / sum_b): the draft row on the target row's scale
+    float inv_sa, inv_sb;
+    float u_draw;        // uniform of the residual / bonus draw
+    int32_t mode;        // 0 none, 1 draw from max(0, p - q), 2 draw from p
+    int32_t valid;       // 0: the row pair is flagged non-finite, its sum of minima is 0
+};
+
 struct FusedShared {
     uint64_t full[FUSED_MAX_SLOTS];                      // one mbarrier per ring slot
-    uint64_t xbar[2];                                    // arrival of the peers' records, by item parity
-    Exchange exch[2][FUSED_MAX_CLUSTER];                 // [item parity][sender rank]
-    Exchange wrec[2][FUSED_MAX_WARPS];                   // [item parity][warp]: the warps' records
-    double tot[10 * FUSED_MAX_WARPS];                    // draw: weight of (vector index i, warp)
-    double pre[10 * FUSED_MAX_WARPS];                    // draw: exclusive prefix of tot
+    uint64_t xbar[3];                                    // arrival of the peers' records, by item mod 3
+    Exchange exch[3][FUSED_MAX_CLUSTER];                 // [item mod 3][sender rank]
+    Exchange wrec[FUSED_MAX_WARPS];                      // the streaming warps' records of the item in pass 1
+    RowConst rc;
+    double tot[FUSED_MAX_WARPS];                         // draw: weight of each streaming warp's range
+    double pre[FUSED_MAX_WARPS];                         // draw: exclusive prefix of tot
     double cta_tot[FUSED_MAX_CLUSTER];                   // draw: weight of each CTA's slice
     double cta_min[16][FUSED_MAX_CLUSTER];               // rank 0: sum of min(p, q) per position and sender
-    float pmin[16][FUSED_MAX_WARPS];                     // sum of min(p, q) per position and warp
+    float pmin[16][FUSED_MAX_WARPS];                     // sum of min(p, q) per position and streaming warp
     const void *table[16];                               // the drafter pointer table
-    // header of the current sequence
-    int32_t h_tok[16];
-    float h_xa[16], h_xb[16], h_u[16], h_ud[FUSED_MAX_POS];
-    int32_t h_t, h_arm;
-    // per-position results of the current sequence
-    int32_t r_acc[16];
-    float r_px[16], r_qx[16];
-    uint32_t r_rowflag[16];
-    int32_t nstar, nlast, token;
-    int32_t dead;       // a wait ran out: later waits do not spin again
+    int32_t token;                                       // rank 0: the drawn token
+    int32_t dead;                                        // a wait ran out: later waits do not spin again
 };
 
 struct FusedGeom {
@@ -194,159 +204,153 @@ __device__ __forceinline__ void wait_bar(FusedShared &sh, uint64_t *bar, uint32_
     atomicOr(status, METASD_STATUS_TIMEOUT);
 }
 
-// Element q of a register array of pairs.
-template <int N>
-__device__ __forceinline__ float elem(const float2 (&a)[N], int q) { return (q & 1) ? a[q >> 1].y : a[q >> 1].x; }
-
-// One row slice from shared memory into registers: e_q = 2^((x_q - m_t) c) with the thread's own
-// maximum m_t, s_t = sum_q e_q.  Vector i of the thread is vector i * nthr + tid of the slice.
-template <typename LT, int VPT>
-__device__ __forceinline__ void load_row(const unsigned char *slot, int my_vecs, int tid, int nthr, float c,
-                                         float2 (&e)[VPT * Logit<LT>::VEC / 2], float &m_t, float &s_t)
+// 16 bytes of logits as pairs of floats.
+template <typename LT>
+__device__ __forceinline__ void unpack2(const uint4 &raw, float2 (&x)[Logit<LT>::VEC / 2])
 {
-    constexpr int NP = VPT * Logit<LT>::VEC / 2;
-    float m = METASD_NEG_BIG;
     if constexpr (sizeof(LT) == 2) {
-        // every lane of a vector outside the slice reads as -inf: weight 0, never the maximum
-        uint32_t w[NP];
+        const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
-        for (int i = 0; i < VPT; ++i) {
-            const int v = i * nthr + tid;
-            uint4 raw = make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);
-            if (v < my_vecs) raw = *reinterpret_cast<const uint4 *>(slot + (size_t)v * 16);
-            w[4 * i] = raw.x; w[4 * i + 1] = raw.y; w[4 * i + 2] = raw.z; w[4 * i + 3] = raw.w;
-        }
-        // the maximum on the packed words, two logits per instruction
-        __nv_bfloat162 m2 = *reinterpret_cast<const __nv_bfloat162 *>(&w[0]);
-#pragma unroll
-        for (int n = 1; n < NP; ++n) m2 = __hmax2(m2, *reinterpret_cast<const __nv_bfloat162 *>(&w[n]));
-        m = fmaxf(m, fmaxf(__low2float(m2), __high2float(m2)));
-#pragma unroll
-        for (int n = 0; n < NP; ++n) e[n] = make_float2(__uint_as_float(w[n] << 16), __uint_as_float(w[n] & 0xFFFF0000u));
+        for (int n = 0; n < 4; ++n) x[n] = make_float2(__uint_as_float(w[n] << 16), __uint_as_float(w[n] & 0xFFFF0000u));
     } else {
-#pragma unroll
-        for (int i = 0; i < VPT; ++i) {
-            const int v = i * nthr + tid;
-            uint4 raw = make_uint4(0xFF800000u, 0xFF800000u, 0xFF800000u, 0xFF800000u);
-            if (v < my_vecs) raw = *reinterpret_cast<const uint4 *>(slot + (size_t)v * 16);
-            e[2 * i] = make_float2(__uint_as_float(raw.x), __uint_as_float(raw.y));
-            e[2 * i + 1] = make_float2(__uint_as_float(raw.z), __uint_as_float(raw.w));
-            m = fmaxf(m, fmaxf(fmaxf(e[2 * i].x, e[2 * i].y), fmaxf(e[2 * i + 1].x, e[2 * i + 1].y)));
-        }
+        x[0] = make_float2(__uint_as_float(raw.x), __uint_as_float(raw.y));
+        x[1] = make_float2(__uint_as_float(raw.z), __uint_as_float(raw.w));
     }
-    const float nm = -m * c;
-    const float2 cc = make_float2(c, c), nn = make_float2(nm, nm);
+}
+
+// Largest of the 16 bytes of logits (NaN entries are ignored).
+template <typename LT>
+__device__ __forceinline__ float vector_max(const uint4 &raw)
+{
+    if constexpr (sizeof(LT) == 2) {
+        const __nv_bfloat162 *w = reinterpret_cast<const __nv_bfloat162 *>(&raw);
+        const __nv_bfloat162 m2 = __hmax2(__hmax2(w[0], w[1]), __hmax2(w[2], w[3]));   // two logits per instruction
+        return fmaxf(__low2float(m2), __high2float(m2));
+    } else {
+        return fmaxf(fmaxf(__uint_as_float(raw.x), __uint_as_float(raw.y)), fmaxf(__uint_as_float(raw.z), __uint_as_float(raw.w)));
+    }
+}
+
+// Pass 1 over one row slice in shared memory: the thread's running maximum m, s = sum 2^((x - m) c) and
+// the first vector that set the maximum.  Thread ct of ncomp takes vectors ct, ct + ncomp, ...
+template <typename LT>
+__device__ __forceinline__ void stats_row(const unsigned char *slot, int my_vecs, int ct, int ncomp, float c, float &m_t,
+                                          float &s_t, int &v_t)
+{
+    constexpr int NP = Logit<LT>::VEC / 2;
+    float m = METASD_NEG_BIG;
     float2 s2 = make_float2(0.f, 0.f);
+    int bv = -1;
+    const float2 cc = make_float2(c, c);
+#pragma unroll 2
+    for (int v = ct; v < my_vecs; v += ncomp) {
+        const uint4 raw = *reinterpret_cast<const uint4 *>(slot + (size_t)v * 16);
+        const float vm = vector_max<LT>(raw);
+        if (vm > m) {   // rare after the first vectors: rescale the sum to the new maximum
+            const float r = ex2((m - vm) * c);
+            s2.x *= r;
+            s2.y *= r;
+            m = vm;
+            bv = v;
+        }
+        const float nm = -m * c;
+        const float2 nn = make_float2(nm, nm);
+        float2 x[NP];
+        unpack2<LT>(raw, x);
 #pragma unroll
-    for (int n = 0; n < NP; ++n) {
-        const float2 y = __ffma2_rn(e[n], cc, nn);
-        e[n] = make_float2(ex2(y.x), ex2(y.y));
-        s2 = __fadd2_rn(s2, e[n]);
+        for (int n = 0; n < NP; ++n) {
+            const float2 y = __ffma2_rn(x[n], cc, nn);
+            s2 = __fadd2_rn(s2, make_float2(ex2(y.x), ex2(y.y)));
+        }
     }
     m_t = m;
     s_t = s2.x + s2.y;
+    v_t = bv;
 }
 
-// First index (in the row) of value m among this thread's logits of a slice, INT_MAX if absent.
-template <typename LT, int VPT>
-__device__ __forceinline__ int first_index_of(const unsigned char *slot, int my_vecs, int tid, int nthr, int vec0, float m)
+// Pass 2 over one row pair in shared memory: sum_v 2^min(ya_v, yb_v) with ya = x_a c + nma, yb = x_b c + nmb_rel,
+// i.e. sum_v min(p_v, q_v) * sum_a.
+template <typename LT>
+__device__ __forceinline__ float min_rows(const unsigned char *slot_a, const unsigned char *slot_b, int my_vecs, int ct,
+                                          int ncomp, float c, float nma, float nmb_rel)
 {
-    constexpr int VEC = Logit<LT>::VEC;
-    int found = INT_MAX;
+    constexpr int NP = Logit<LT>::VEC / 2;
+    const float2 cc = make_float2(c, c), na = make_float2(nma, nma), nb = make_float2(nmb_rel, nmb_rel);
+    float2 acc = make_float2(0.f, 0.f);
+#pragma unroll 2
+    for (int v = ct; v < my_vecs; v += ncomp) {
+        const uint4 ra = *reinterpret_cast<const uint4 *>(slot_a + (size_t)v * 16);
+        const uint4 rb = *reinterpret_cast<const uint4 *>(slot_b + (size_t)v * 16);
+        float2 xa[NP], xb[NP];
+        unpack2<LT>(ra, xa);
+        unpack2<LT>(rb, xb);
 #pragma unroll
-    for (int i = VPT - 1; i >= 0; --i) {
-        const int v = i * nthr + tid;
-        if (v < my_vecs) {
-            float x[VEC];
-            Logit<LT>::unpack(*reinterpret_cast<const uint4 *>(slot + (size_t)v * 16), x);
-#pragma unroll
-            for (int q = VEC - 1; q >= 0; --q)
-                if (x[q] == m) found = (vec0 + v) * VEC + q;
+        for (int n = 0; n < NP; ++n) {
+            const float2 ya = __ffma2_rn(xa[n], cc, na), yb = __ffma2_rn(xb[n], cc, nb);
+            acc = __fadd2_rn(acc, make_float2(ex2(fminf(ya.x, yb.x)), ex2(fminf(ya.y, yb.y))));
         }
     }
-    return found;
+    return acc.x + acc.y;
 }
 
-// Merges up to 32 records held one per lane (lanes >= n hold nothing): row maxima, row sums relative
-// to them, the first arg-max of the target row, and each lane's own rescaling factors.
-struct Merged {
-    float Ma, Sa, Mb, Sb;
-    int idx;
-    float ta, tb;   // this lane's 2^((m_lane - M) c)
-};
-__device__ __forceinline__ Merged merge_records(const Exchange *rec, int n, int lane, float c)
+// Weights of the draw for one vector: mode 1 = max(0, p - q) (correction), mode 2 = p (bonus).
+template <typename LT>
+__device__ __forceinline__ void draw_weights(const unsigned char *slot_a, const unsigned char *slot_b, int v, int mode,
+                                             float c, const RowConst &rc, float (&w)[Logit<LT>::VEC])
 {
-    float ma = METASD_NEG_BIG, sa = 0.f, mb = METASD_NEG_BIG, sb = 0.f;
-    int ia = INT_MAX;
-    if (lane < n) {
-        const Exchange x = rec[lane];
-        ma = x.max_a; sa = x.sum_a; mb = x.max_b; sb = x.sum_b; ia = x.idx_a;
+    constexpr int VEC = Logit<LT>::VEC;
+    float xa[VEC], xb[VEC];
+    Logit<LT>::unpack(*reinterpret_cast<const uint4 *>(slot_a + (size_t)v * 16), xa);
+    if (mode == 1) Logit<LT>::unpack(*reinterpret_cast<const uint4 *>(slot_b + (size_t)v * 16), xb);
+#pragma unroll
+    for (int q = 0; q < VEC; ++q) {
+        const float pv = ex2(fmaf(xa[q], c, rc.nma)) * rc.inv_sa;
+        if (mode == 1) {
+            const float qv = ex2(fmaf(xb[q], c, rc.nmb)) * rc.inv_sb;
+            w[q] = fmaxf(pv - qv, 0.f);
+        } else {
+            w[q] = pv;
+        }
     }
-    Merged r;
-    r.Ma = warp_max_f(ma);
-    r.Mb = warp_max_f(mb);
-    r.ta = ex2((ma - r.Ma) * c);
-    r.tb = ex2((mb - r.Mb) * c);
-    r.Sa = warp_sum_f(sa * r.ta);
-    r.Sb = warp_sum_f(sb * r.tb);
-    r.idx = __reduce_min_sync(0xFFFFFFFFu, (lane < n && ma == r.Ma) ? ia : INT_MAX);
-    return r;
 }
 
-// Weight of element q in the draw: mode 1 = max(0, p - q) (correction), mode 2 = p (bonus).
-__device__ __forceinline__ float draw_weight(int mode, float ea, float fa, float eb, float fb)
-{
-    const float pv = ea * fa;
-    return mode == 1 ? fmaxf(pv - eb * fb, 0.f) : pv;
-}
-
-// Inverse CDF in token order over one row (pair) that lives in the registers of the whole cluster:
-// the smallest v with sum_{w <= v} weight_w > u * total.  Token order is (rank, vector i, thread, lane
-// of the vector).  Totals and offsets are carried in fp64.  Returns false (for every thread of the
+// Inverse CDF in token order over one row (pair) that lives in the shared memory of the whole cluster:
+// the smallest v with sum_{w <= v} weight_w > u * total.  Every streaming warp owns a contiguous range
+// of its CTA's slice; totals and offsets are carried in fp64.  Returns false (for every thread of the
 // cluster alike) when the row has no mass; otherwise the token lands in sh.token of rank 0.
-template <int VPT, int VEC>
-__device__ bool cluster_draw(FusedShared &sh, const float2 (&ea)[VPT * VEC / 2], const float2 (&eb)[VPT * VEC / 2], float fa,
-                             float fb, int mode, float u, int rank, int csize, int vec0, int nthr)
+template <typename LT>
+__device__ bool cluster_draw(FusedShared &sh, const unsigned char *slot_a, const unsigned char *slot_b, int mode, float c,
+                             int my_vecs, int vec0, int rank, int csize, int ncw)
 {
+    constexpr int VEC = Logit<LT>::VEC;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int nw = nthr >> 5, ne = VPT * nw;
-    float vs[VPT];
+    const RowConst rc = sh.rc;
+    const int per_warp = (my_vecs + ncw - 1) / ncw;
+    const int cw = warp - 1;   // streaming warp index; the control warp has none
+    const int v0 = cw >= 0 ? min(cw * per_warp, my_vecs) : 0, v1 = cw >= 0 ? min(v0 + per_warp, my_vecs) : 0;
+    if (cw >= 0) {
+        double acc = 0.0;
+        for (int v = v0 + lane; v < v1; v += 32) {
+            float w[VEC];
+            draw_weights<LT>(slot_a, slot_b, v, mode, c, rc, w);
+            float s = 0.f;
 #pragma unroll
-    for (int i = 0; i < VPT; ++i) {
-        float s = 0.f;
-#pragma unroll
-        for (int q = 0; q < VEC; ++q) s += draw_weight(mode, elem(ea, i * VEC + q), fa, elem(eb, i * VEC + q), fb);
-        vs[i] = s;
-    }
-    if (tid == 0) { sh.nstar = INT_MAX; sh.nlast = -1; }
-#pragma unroll
-    for (int i = 0; i < VPT; ++i) {
-        const double d = warp_sum((double)vs[i]);
-        if (lane == 0) sh.tot[i * nw + warp] = d;
+            for (int q = 0; q < VEC; ++q) s += w[q];
+            acc += (double)s;
+        }
+        acc = warp_sum(acc);
+        if (lane == 0) sh.tot[cw] = acc;
     }
     __syncthreads();
     if (warp == 0) {
-        // exclusive prefix over the ne entries, `per` consecutive entries per lane
-        const int per = (ne + 31) >> 5;
-        double loc[5], sum = 0.0;
-#pragma unroll
-        for (int q = 0; q < 5; ++q) {
-            const int n = lane * per + q;
-            loc[q] = (q < per && n < ne) ? sh.tot[n] : 0.0;
-            sum += loc[q];
-        }
-        double incl = sum;
+        const double t = lane < ncw ? sh.tot[lane] : 0.0;
+        double incl = t;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
-            const double t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-            if (lane >= o) incl += t;
+            const double x = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+            if (lane >= o) incl += x;
         }
-        double run = incl - sum;
-#pragma unroll
-        for (int q = 0; q < 5; ++q) {
-            const int n = lane * per + q;
-            if (q < per && n < ne) { sh.pre[n] = run; run += loc[q]; }
-        }
+        if (lane < ncw) sh.pre[lane] = incl - t;
         const double total = __shfl_sync(0xFFFFFFFFu, incl, 31);
         if (lane < csize) st_cluster(map_to_rank(smem_addr(&sh.cta_tot[rank]), lane), total);
     }
@@ -360,7 +364,7 @@ __device__ bool cluster_draw(FusedShared &sh, const float2 (&ea)[VPT * VEC / 2],
         R += t;
     }
     if (!(R > 0.0)) return false;
-    const double thr = (double)u * R;
+    const double thr = (double)rc.u_draw * R;
     int rstar = -1;
     {
         double run = 0.0;
@@ -371,54 +375,90 @@ __device__ bool cluster_draw(FusedShared &sh, const float2 (&ea)[VPT * VEC / 2],
         }
     }
     if (rstar < 0) rstar = rlast;   // rounding left the total a hair under the threshold
-    if (rank == rstar) {
+    if (rank == rstar && cw >= 0) {
         const double th = thr - mybase;
-        if (tid < ne) {
-            const double t = sh.tot[tid];
-            if (t > 0.0) atomicMax(&sh.nlast, tid);
-            if (sh.pre[tid] + t > th) atomicMin(&sh.nstar, tid);
-        }
-        __syncthreads();
-        const int n = sh.nstar != INT_MAX ? sh.nstar : sh.nlast;
-        const int istar = n / nw, wstar = n - istar * nw;
-        if (warp == wstar) {
-            float v = 0.f;
+        // the warp whose range holds the crossing; rounding may leave none: then the last warp with mass
+        const double t = lane < ncw ? sh.tot[lane] : 0.0;
+        const double pr = lane < ncw ? sh.pre[lane] : 0.0;
+        const unsigned crossing = __ballot_sync(0xFFFFFFFFu, lane < ncw && pr + t > th);
+        const unsigned mass = __ballot_sync(0xFFFFFFFFu, lane < ncw && t > 0.0);
+        const int wstar = crossing ? __ffs(crossing) - 1 : 31 - __clz(mass);
+        if (cw == wstar) {
+            int found = -1, last_pos = -1;
+            double run_base = sh.pre[wstar];
+            for (int i0 = v0; i0 < v1 && found < 0; i0 += 32) {
+                const int v = i0 + lane;
+                float w[VEC];
 #pragma unroll
-            for (int i = 0; i < VPT; ++i)
-                if (i == istar) v = vs[i];
-            const double dv = (double)v;
-            double incl = dv;
+                for (int q = 0; q < VEC; ++q) w[q] = 0.f;
+                if (v < v1) draw_weights<LT>(slot_a, slot_b, v, mode, c, rc, w);
+                float s = 0.f;
 #pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const double t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-                if (lane >= o) incl += t;
-            }
-            const double pre = sh.pre[n];
-            const unsigned crossing = __ballot_sync(0xFFFFFFFFu, pre + incl > th);
-            const unsigned mass = __ballot_sync(0xFFFFFFFFu, v > 0.f);
-            const int src = crossing ? __ffs(crossing) - 1 : (mass ? 31 - __clz(mass) : 0);
-            if (lane == src) {
-                double cum = pre + incl - dv;
-                int tok_q = -1, last_q = -1;
+                for (int q = 0; q < VEC; ++q) s += w[q];
+                double incl = (double)s;
 #pragma unroll
-                for (int i = 0; i < VPT; ++i) {
-                    if (i == istar) {
+                for (int o = 1; o < 32; o <<= 1) {
+                    const double x = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+                    if (lane >= o) incl += x;
+                }
+                const unsigned ballot = __ballot_sync(0xFFFFFFFFu, run_base + incl > th);
+#pragma unroll
+                for (int q = 0; q < VEC; ++q)
+                    if (w[q] > 0.f) last_pos = (vec0 + v) * VEC + q;
+                if (ballot) {
+                    const int src = __ffs(ballot) - 1;
+                    if (lane == src) {
+                        double cum = run_base + incl - (double)s;
+                        int tok = -1;
 #pragma unroll
                         for (int q = 0; q < VEC; ++q) {
-                            const float w = draw_weight(mode, elem(ea, i * VEC + q), fa, elem(eb, i * VEC + q), fb);
-                            cum += (double)w;
-                            if (w > 0.f) last_q = q;
-                            if (tok_q < 0 && cum > th) tok_q = q;
+                            cum += (double)w[q];
+                            if (tok < 0 && cum > th) tok = (vec0 + v) * VEC + q;
                         }
+                        // the vector's own sum crossed, so an element does unless rounding interferes
+                        if (tok < 0) {
+#pragma unroll
+                            for (int q = 0; q < VEC; ++q)
+                                if (w[q] > 0.f) tok = (vec0 + v) * VEC + q;
+                        }
+                        found = tok;
                     }
+                    found = __shfl_sync(0xFFFFFFFFu, found, src);
                 }
-                if (tok_q < 0) tok_q = last_q;
-                const int token = tok_q < 0 ? -1 : (vec0 + istar * nthr + tid) * VEC + tok_q;
-                st_cluster(map_to_rank(smem_addr(&sh.token), 0), (int32_t)token);
+                run_base += __shfl_sync(0xFFFFFFFFu, incl, 31);
             }
+            if (found < 0) {   // rounding left the running sum a hair under the threshold
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) last_pos = max(last_pos, __shfl_xor_sync(0xFFFFFFFFu, last_pos, o));
+                found = last_pos;
+            }
+            if (lane == 0) st_cluster(map_to_rank(smem_addr(&sh.token), 0), (int32_t)found);
         }
     }
     return true;
+}
+
+// Merges up to 32 records held one per lane (lanes >= n hold nothing): row maxima, row sums relative
+// to them and the first arg-max of the target row.
+struct Merged {
+    float Ma, Sa, Mb, Sb;
+    int idx;
+};
+__device__ __forceinline__ Merged merge_records(const Exchange *rec, int n, int lane, float c)
+{
+    float ma = METASD_NEG_BIG, sa = 0.f, mb = METASD_NEG_BIG, sb = 0.f;
+    int ia = INT_MAX;
+    if (lane < n) {
+        const Exchange x = rec[lane];
+        ma = x.max_a; sa = x.sum_a; mb = x.max_b; sb = x.sum_b; ia = x.idx_a;
+    }
+    Merged r;
+    r.Ma = warp_max_f(ma);
+    r.Mb = warp_max_f(mb);
+    r.Sa = warp_sum_f(sa * ex2((ma - r.Ma) * c));
+    r.Sb = warp_sum_f(sb * ex2((mb - r.Mb) * c));
+    r.idx = __reduce_min_sync(0xFFFFFFFFu, (lane < n && ma == r.Ma) ? ia : INT_MAX);
+    return r;
 }
 
 // Bandit update and next selection by one warp, lane i = drafter i (Algorithm 2 lines 7-10; Discounted
@@ -488,16 +528,17 @@ __device__ void warp_bandit(const VerifyParams &p, int b, int t, int arm, double
 // ---------------------------------------------------------------------------------------------
 // The kernel
 // ---------------------------------------------------------------------------------------------
-template <typename LT, int VPT>
+template <typename LT>
 __global__ void __launch_bounds__(FUSED_MAX_THREADS, 1) fused_round_kernel(const VerifyParams p, const FusedGeom g)
 {
     constexpr int VEC = Logit<LT>::VEC;
-    constexpr int NP = VPT * VEC / 2;
     extern __shared__ __align__(128) unsigned char ring[];
     __shared__ FusedShared sh;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int nthr = blockDim.x, nw = nthr >> 5;
+    const int ncw = (blockDim.x >> 5) - 1;            // streaming warps
+    const int ncomp = ncw * 32, ct = tid - 32;        // streaming threads and this thread's index among them
+    const bool control = warp == 0;
     const int rank = (int)cluster_rank(), csize = (int)cluster_size();
     const int cid = (int)cluster_id(), ncl = (int)cluster_count();
     const int k = p.k, V = p.V;
@@ -509,8 +550,7 @@ __global__ void __launch_bounds__(FUSED_MAX_THREADS, 1) fused_round_kernel(const
 
     if (tid == 0) {
         for (int s = 0; s < g.n_slot; ++s) mbar_init(&sh.full[s], 1);
-        mbar_init(&sh.xbar[0], 1);
-        mbar_init(&sh.xbar[1], 1);
+        for (int s = 0; s < 3; ++s) mbar_init(&sh.xbar[s], 1);
         sh.dead = 0;
         sh.token = -1;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -518,9 +558,11 @@ __global__ void __launch_bounds__(FUSED_MAX_THREADS, 1) fused_round_kernel(const
     if (tid < 16) sh.table[tid] = (p.drafter_ptrs && tid < p.K) ? p.drafter_ptrs[tid] : nullptr;
     cluster_sync_all();   // every CTA of the cluster is running, its barriers initialised, before a peer writes to it
 
+    const int n_seq = cid < p.batch ? (p.batch - cid + ncl - 1) / ncl : 0;   // sequences of this cluster
+    const int n_items = n_seq * (k + 1);
+
     // ---- producer (thread 0): the order of loads is sequence-major, position, target then draft
     int ld_b = cid, ld_j = 0, ld_row = 0, ld_slot = 0, ld_arm_next = 0;
-    uint32_t ld_issued = 0, consumed = 0;
     const unsigned char *ld_draft = nullptr;
     auto draft_base = [&](int arm) -> const unsigned char * {
         return reinterpret_cast<const unsigned char *>(p.draft ? p.draft : sh.table[arm & 15]);
@@ -540,7 +582,6 @@ __global__ void __launch_bounds__(FUSED_MAX_THREADS, 1) fused_round_kernel(const
             mbar_arrive_expect_tx(bar, my_bytes);
             bulk_load(ring + (size_t)ld_slot * g.slot_bytes, src, my_bytes, bar);
         }
-        ++ld_issued;
         ld_slot = ld_slot + 1 == g.n_slot ? 0 : ld_slot + 1;
         if (ld_row == 0 && ld_j < k) {
             ld_row = 1;
@@ -556,14 +597,14 @@ __global__ void __launch_bounds__(FUSED_MAX_THREADS, 1) fused_round_kernel(const
             }
         }
     };
-    if (tid == 0 && cid < p.batch) {
+    if (tid == 0 && n_seq > 0) {
         ld_draft = draft_base(p.draft ? 0 : p.st.arm[cid]);
         if (!p.draft && cid + ncl < p.batch) ld_arm_next = p.st.arm[cid + ncl];
         for (int s = 0; s < g.n_slot; ++s) issue_one();
     }
 
-    // ---- header of a sequence (warp 0, lane j = position j): round counter, arm, drafted token and
-    // its two logits.  Fetched one sequence ahead, in three steps spread over the item loop.
+    // ---- control warp, lane j = position j: header of a sequence (round counter, arm, drafted token, its
+    // two logits), fetched one sequence ahead in three steps spread over the items
     int nx_t = 0, nx_arm = 0, nx_tok = -1;
     float nx_xa = 0.f, nx_xb = 0.f;
     auto fetch_step = [&](int b, int step) {
@@ -586,229 +627,238 @@ __global__ void __launch_bounds__(FUSED_MAX_THREADS, 1) fused_round_kernel(const
             }
         }
     };
-    if (warp == 0 && cid < p.batch) {
+    if (control && n_seq > 0) {
         fetch_step(cid, 0);
         fetch_step(cid, 1);
         fetch_step(cid, 2);
     }
+    // header and results of the sequence in pass 2 (control warp registers, lane j = position j)
+    int h_t = 0, h_arm = 0, h_tok = -1, r_acc = 0;
+    float h_xa = 0.f, h_xb = 0.f, h_u = 0.f, h_ud = 0.f, r_px = 0.f, r_qx = 0.f;
+    uint32_t r_rowflag = 0, seq_flags = 0;
+    int n_acc = -1, token = -1;   // n_acc < 0: no rejection yet
+    bool drew = false;            // the token sits in sh.token of rank 0
 
-    int cs = 0;              // ring slot the consumers read next
-    uint32_t cpar = 0;       // and its phase parity
-    uint32_t item = 0;       // items done by this cluster: bit 0 selects the exchange buffers, bit 1 their phase
+    // cursors: pass 1 consumes ring slots c1, pass 2 (one item behind) reads slots c2 and then frees them
+    int j1 = 0, c1 = 0, b2 = cid, j2 = 0, c2 = 0;
+    uint32_t c1par = 0;
+    int u1 = 0, u2 = 0;            // item mod 3 of pass 1 / pass 2: which exchange buffer
+    uint32_t x2par = 0;            // phase parity of xbar[u2]
 
-    for (int b = cid; b < p.batch; b += ncl) {
-        // ---- publish the header of sequence b
-        if (warp == 0) {
-            if (lane == 0) { sh.h_t = nx_t; sh.h_arm = nx_arm; }
-            if (lane <= k) {
-                const uint4 w = round_words(p.seed, p.sequence_base + (uint32_t)b, (uint32_t)nx_t, (uint32_t)lane);
-                sh.h_ud[lane] = uniform24(w.y);
-                if (lane < k) {
-                    sh.h_u[lane] = uniform24(w.x);
-                    sh.h_tok[lane] = nx_tok;
-                    sh.h_xa[lane] = nx_xa;
-                    sh.h_xb[lane] = nx_xb;
+    for (int step = 0; step <= n_items; ++step) {
+        const bool do1 = step < n_items, do2 = step >= 1;
+        const bool pair1 = j1 < k, pair2 = j2 < k;
+        const unsigned char *a2 = ring + (size_t)c2 * g.slot_bytes;
+        const unsigned char *d2 = ring + (size_t)(c2 + 1 == g.n_slot ? 0 : c2 + 1) * g.slot_bytes;
+
+        if (control) {
+            // ---- expect one record of 32 bytes from every CTA of the cluster (this one included) for pass 1's item
+            if (do1 && lane == 0 && !*(volatile int32_t *)&sh.dead)
+                mbar_arrive_expect_tx(&sh.xbar[u1], (uint32_t)csize * EXCHANGE_BYTES);
+            if (do2) {
+                // ---- pass 2's item: merged records, flags, the accept test of Algorithm 4 (lines 7-8), what to draw
+                if (j2 == 0) {   // a new sequence enters pass 2
+                    h_t = nx_t; h_arm = nx_arm; h_tok = nx_tok; h_xa = nx_xa; h_xb = nx_xb;
+                    const uint4 w = round_words(p.seed, p.sequence_base + (uint32_t)b2, (uint32_t)h_t, (uint32_t)lane);
+                    h_u = uniform24(w.x);
+                    h_ud = uniform24(w.y);
+                    n_acc = -1; token = -1; drew = false; seq_flags = 0; r_acc = 0; r_px = 0.f; r_qx = 0.f; r_rowflag = 0;
                 }
-            }
-        }
-        const int b_next = b + ncl;
-        int n_acc = -1;          // undecided
-        int token = -1;
-        bool drew = false;       // the token sits in sh.token of rank 0
-        uint32_t seq_flags = 0;
-
-        for (int j = 0; j <= k; ++j, ++item) {
-            const bool pair = j < k;
-            const int par = item & 1;
-            if (warp == 0) {
+                const int b_next = b2 + ncl;
                 if (b_next < p.batch) {
-                    if (j == 0) fetch_step(b_next, 0);
-                    if (j == 1) fetch_step(b_next, 1);
-                    if (j == (k < 2 ? k : 2)) fetch_step(b_next, 2);
+                    if (j2 == 0) fetch_step(b_next, 0);
+                    if (j2 == 1) fetch_step(b_next, 1);
+                    if (j2 == (k < 2 ? k : 2)) fetch_step(b_next, 2);
                 }
-                // expect one record of 32 bytes from every CTA of the cluster (this one included)
-                if (lane == 0 && !*(volatile int32_t *)&sh.dead)
-                    mbar_arrive_expect_tx(&sh.xbar[par], (uint32_t)csize * EXCHANGE_BYTES);
+                wait_bar(sh, &sh.xbar[u2], x2par, p.status);
+                const Merged mg = merge_records(sh.exch[u2], csize, lane, c);
+                // NaN or +Inf anywhere makes the sum NaN; an all -Inf row leaves it 0
+                const bool bad_a = !(mg.Sa > 0.f) || !(mg.Sa < INFINITY) || !(mg.Ma < INFINITY);
+                const bool bad_b = pair2 && (!(mg.Sb > 0.f) || !(mg.Sb < INFINITY) || !(mg.Mb < INFINITY));
+                const uint32_t rowflag = (bad_a || bad_b) ? METASD_STATUS_NONFINITE : 0u;
+                const float nma = -mg.Ma * c, nmb = -mg.Mb * c;
+                bool accepted = false;
+                if (pair2) {
+                    // lane j2 holds this position's token; every lane evaluates it on the broadcast values
+                    const int x = __shfl_sync(0xFFFFFFFFu, h_tok, j2);
+                    const float xa = __shfl_sync(0xFFFFFFFFu, h_xa, j2), xb = __shfl_sync(0xFFFFFFFFu, h_xb, j2);
+                    const float u = __shfl_sync(0xFFFFFFFFu, h_u, j2);
+                    float p_x = 0.f, q_x = 0.f;
+                    uint32_t fl = rowflag;
+                    if (!rowflag) {
+                        if (x < 0 || x >= V) {
+                            fl |= METASD_STATUS_TOKEN_OOR;
+                        } else {
+                            p_x = ex2(fmaf(xa, c, nma)) / mg.Sa;
+                            q_x = ex2(fmaf(xb, c, nmb)) / mg.Sb;
+                            if (p.greedy) {
+                                accepted = x == mg.idx;
+                            } else {
+                                if (q_x == 0.f) fl |= METASD_STATUS_Q_ZERO;
+                                accepted = u * q_x < p_x;   // u < min(1, p/q) without the division
+                            }
+                        }
+                    }
+                    seq_flags |= fl;
+                    if (lane == j2) { r_acc = accepted ? 1 : 0; r_px = p_x; r_qx = q_x; r_rowflag = rowflag; }
+                }
+                // first rejection (Algorithm 4, "exit for loop") or the bonus position: the next token comes from here
+                int mode = 0;
+                if (n_acc < 0) {
+                    if (pair2 && !accepted) { n_acc = j2; mode = 1; }
+                    if (!pair2) { n_acc = k; mode = 2; seq_flags |= rowflag; }
+                    if (mode) {
+                        if (rowflag) {
+                            mode = 0;
+                        } else if (p.greedy) {
+                            token = mg.idx;
+                            mode = 0;
+                        }
+                    }
+                }
+                const float ud = __shfl_sync(0xFFFFFFFFu, h_ud, j2);
+                if (lane == 0) {
+                    RowConst rc;
+                    rc.nma = nma;
+                    rc.nmb = nmb;
+                    // q_v / p_v = 2^(yb - ya) sum_a / sum_b: the ratio of the sums folds into the draft row's offset
+                    rc.nmb_rel = nmb + log2f(mg.Sa / mg.Sb);
+                    rc.inv_sa = 1.0f / mg.Sa;
+                    rc.inv_sb = 1.0f / mg.Sb;
+                    rc.u_draw = ud;
+                    rc.mode = mode;
+                    rc.valid = rowflag ? 0 : 1;
+                    sh.rc = rc;
+                }
             }
-
-            // ---- this item's slices: shared memory -> registers, exponentials relative to the thread maximum,
-            //      then the warp's record: maxima, sums relative to them, first arg-max of the target row
-            float2 ea[NP], eb[NP];
-            float mta, mtb = METASD_NEG_BIG;
+        } else if (do1) {
+            // ---- pass 1: statistics of this item's row slices out of shared memory
             Exchange wr;
-            {
-                float sta;
-                const unsigned char *slot = ring + (size_t)cs * g.slot_bytes;
-                wait_bar(sh, &sh.full[cs], cpar, p.status);
-                load_row<LT, VPT>(slot, my_vecs, tid, nthr, c, ea, mta, sta);
-                if (++cs == g.n_slot) { cs = 0; cpar ^= 1u; }
-                wr.max_a = warp_max_f(mta);
-                wr.sum_a = warp_sum_f(sta * ex2((mta - wr.max_a) * c));
-                int cand = INT_MAX;
-                if (p.greedy && mta == wr.max_a && mta > METASD_NEG_BIG)
-                    cand = first_index_of<LT, VPT>(slot, my_vecs, tid, nthr, vec0, mta);
-                wr.idx_a = p.greedy ? __reduce_min_sync(0xFFFFFFFFu, cand) : INT_MAX;
-            }
-            if (pair) {
-                float stb;
-                wait_bar(sh, &sh.full[cs], cpar, p.status);
-                load_row<LT, VPT>(ring + (size_t)cs * g.slot_bytes, my_vecs, tid, nthr, c, eb, mtb, stb);
-                if (++cs == g.n_slot) { cs = 0; cpar ^= 1u; }
-                wr.max_b = warp_max_f(mtb);
-                wr.sum_b = warp_sum_f(stb * ex2((mtb - wr.max_b) * c));
-            } else {
+            float m_t, s_t;
+            int v_t, v_dummy;
+            const unsigned char *slot = ring + (size_t)c1 * g.slot_bytes;
+            wait_bar(sh, &sh.full[c1], c1par, p.status);
+            stats_row<LT>(slot, my_vecs, ct, ncomp, c, m_t, s_t, v_t);
+            wr.max_a = warp_max_f(m_t);
+            wr.sum_a = warp_sum_f(s_t * ex2((m_t - wr.max_a) * c));
+            int cand = INT_MAX;
+            if (p.greedy && m_t == wr.max_a && v_t >= 0) {   // first index of the maximum inside the vector that set it
+                float x[VEC];
+                Logit<LT>::unpack(*reinterpret_cast<const uint4 *>(slot + (size_t)v_t * 16), x);
 #pragma unroll
-                for (int n = 0; n < NP; ++n) eb[n] = make_float2(0.f, 0.f);
-                wr.max_b = METASD_NEG_BIG;
-                wr.sum_b = 0.f;
+                for (int q = VEC - 1; q >= 0; --q)
+                    if (x[q] == m_t) cand = (vec0 + v_t) * VEC + q;
+            }
+            wr.idx_a = p.greedy ? __reduce_min_sync(0xFFFFFFFFu, cand) : INT_MAX;
+            wr.max_b = METASD_NEG_BIG;
+            wr.sum_b = 0.f;
+            if (pair1) {
+                const int cb = c1 + 1 == g.n_slot ? 0 : c1 + 1;
+                wait_bar(sh, &sh.full[cb], cb == 0 ? c1par ^ 1u : c1par, p.status);
+                stats_row<LT>(ring + (size_t)cb * g.slot_bytes, my_vecs, ct, ncomp, c, m_t, s_t, v_dummy);
+                wr.max_b = warp_max_f(m_t);
+                wr.sum_b = warp_sum_f(s_t * ex2((m_t - wr.max_b) * c));
             }
             if (lane == 0) {
                 wr.pad[0] = wr.pad[1] = wr.pad[2] = 0;
-                sh.wrec[par][warp] = wr;
+                sh.wrec[warp - 1] = wr;
             }
-            __syncthreads();
+        }
+        __syncthreads();   // (C) the warps' records and pass 2's row constants are in shared memory
 
-            // ---- the slots of this item are free: refill them
-            if (tid == 0) {
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                consumed += pair ? 2u : 1u;
-                issue_one();
-                if (pair) issue_one();
-            }
-            // ---- the CTA's record goes to every CTA of the cluster (asynchronous stores that complete on
-            //      the receiver's barrier); then wait for all the records addressed to this CTA
-            if (warp == 0) {
-                const Merged mc = merge_records(sh.wrec[par], nw, lane, c);
+        if (control) {
+            // ---- the CTA's record of pass 1's item goes to every CTA of the cluster
+            if (do1) {
+                const Merged mc = merge_records(sh.wrec, ncw, lane, c);
                 if (lane < csize) {
-                    const uint32_t dst = map_to_rank(smem_addr(&sh.exch[par][rank]), (uint32_t)lane);
-                    const uint32_t bar = map_to_rank(smem_addr(&sh.xbar[par]), (uint32_t)lane);
+                    const uint32_t dst = map_to_rank(smem_addr(&sh.exch[u1][rank]), (uint32_t)lane);
+                    const uint32_t bar = map_to_rank(smem_addr(&sh.xbar[u1]), (uint32_t)lane);
                     st_async_16(dst, bar, __float_as_uint(mc.Ma), __float_as_uint(mc.Sa), __float_as_uint(mc.Mb),
                                 __float_as_uint(mc.Sb));
                     st_async_16(dst + 16, bar, (uint32_t)mc.idx, 0u, 0u, 0u);
                 }
             }
-            wait_bar(sh, &sh.xbar[par], (item >> 1) & 1u, p.status);
-            const Merged mg = merge_records(sh.exch[par], csize, lane, c);
-            const float Ma = mg.Ma, Sa = mg.Sa, Mb = mg.Mb, Sb = mg.Sb;
-            const int argidx = mg.idx;
-
-            // NaN or +Inf anywhere makes the sum NaN; an all -Inf row leaves it 0
-            const bool bad_a = !(Sa > 0.f) || !(Sa < INFINITY) || !(Ma < INFINITY);
-            const bool bad_b = pair && (!(Sb > 0.f) || !(Sb < INFINITY) || !(Mb < INFINITY));
-            const uint32_t rowflag = (bad_a || bad_b) ? METASD_STATUS_NONFINITE : 0u;
-            // p_v = e_v * fa with fa = 2^((m_t - M) c) / S
-            const float fa = rowflag ? 0.f : ex2((mta - Ma) * c) / Sa;
-            const float fb = (rowflag || !pair) ? 0.f : ex2((mtb - Mb) * c) / Sb;
-
-            // ---- sum_v min(p_v, q_v) of this warp's logits
-            bool accepted = false;
-            if (pair) {
-                float2 acc2 = make_float2(0.f, 0.f);
-                const float2 fa2 = make_float2(fa, fa), fb2 = make_float2(fb, fb);
-#pragma unroll
-                for (int n = 0; n < NP; ++n) {
-                    const float2 pv = __fmul2_rn(ea[n], fa2), qv = __fmul2_rn(eb[n], fb2);
-                    acc2 = __fadd2_rn(acc2, make_float2(fminf(pv.x, qv.x), fminf(pv.y, qv.y)));
-                }
-                const float acc = warp_sum_f(acc2.x + acc2.y);
-                if (lane == 0) sh.pmin[j][warp] = acc;
-
-                // ---- the accept test of Algorithm 4 (lines 7-8), evaluated alike by every thread of the cluster
-                const int x = sh.h_tok[j];
-                float p_x = 0.f, q_x = 0.f;
-                uint32_t fl = rowflag;
-                if (!rowflag) {
-                    if (x < 0 || x >= V) {
-                        fl |= METASD_STATUS_TOKEN_OOR;
-                    } else {
-                        p_x = ex2(fmaf(sh.h_xa[j], c, -Ma * c)) / Sa;
-                        q_x = ex2(fmaf(sh.h_xb[j], c, -Mb * c)) / Sb;
-                        if (p.greedy) {
-                            accepted = x == argidx;
-                        } else {
-                            if (q_x == 0.f) fl |= METASD_STATUS_Q_ZERO;
-                            accepted = sh.h_u[j] * q_x < p_x;   // u < min(1, p/q) without the division
-                        }
-                    }
-                }
-                seq_flags |= fl;
-                if (tid == 0) {
-                    sh.r_acc[j] = accepted ? 1 : 0;
-                    sh.r_px[j] = p_x;
-                    sh.r_qx[j] = q_x;
-                    sh.r_rowflag[j] = rowflag;
-                }
-            }
-
-            // ---- first rejection (Algorithm 4, "exit for loop") or the bonus position: emit the next token
-            int mode = 0;
-            if (n_acc < 0) {
-                if (pair && !accepted) { n_acc = j; mode = 1; }
-                if (!pair) { n_acc = k; mode = 2; seq_flags |= rowflag; }
-                if (mode) {
-                    if (rowflag) {
-                        mode = 0;
-                    } else if (p.greedy) {
-                        token = argidx;
-                        mode = 0;
-                    }
-                }
-            }
+        } else if (do2 && pair2) {
+            // ---- pass 2: sum_v min(p_v, q_v) of this warp's logits
+            const RowConst rc = sh.rc;
+            float acc = 0.f;
+            if (rc.valid) acc = min_rows<LT>(a2, d2, my_vecs, ct, ncomp, c, rc.nma, rc.nmb_rel) * rc.inv_sa;
+            acc = warp_sum_f(acc);
+            if (lane == 0) sh.pmin[j2][warp - 1] = acc;
+        }
+        if (do2) {
+            const int mode = sh.rc.mode;   // alike in every thread of the cluster
             if (mode) {
-                const float u = sh.h_ud[j];
-                bool ok = cluster_draw<VPT, VEC>(sh, ea, eb, fa, fb, mode, u, rank, csize, vec0, nthr);
+                bool ok = cluster_draw<LT>(sh, a2, d2, mode, c, my_vecs, vec0, rank, csize, ncw);
                 if (!ok && mode == 1)   // p == q in fp32 yet rejected: draw from p
-                    ok = cluster_draw<VPT, VEC>(sh, ea, eb, fa, fb, 2, u, rank, csize, vec0, nthr);
+                    ok = cluster_draw<LT>(sh, a2, d2, 2, c, my_vecs, vec0, rank, csize, ncw);
                 drew = ok;
             }
+            if (!pair2) {
+                // ---- end of the sequence: gather sum_v min(p, q) per position in rank 0
+                __syncthreads();
+                if (control && lane < k) {
+                    double s = 0.0;
+                    for (int w = 0; w < ncw; ++w) s += (double)sh.pmin[lane][w];
+                    st_cluster(map_to_rank(smem_addr(&sh.cta_min[lane][rank]), 0), s);
+                }
+                cluster_sync_all();
+                if (rank == 0 && control) {
+                    double smin = 0.0;
+                    if (lane < k) {
+                        for (int r = 0; r < csize; ++r) smin += sh.cta_min[lane][r];
+                        if (r_rowflag) smin = 0.0;
+                    }
+                    double sum_align = 0.0;
+                    for (int j = 0; j < k; ++j) sum_align += __shfl_sync(0xFFFFFFFFu, smin, j);
+                    // Definition 2: 1 - mean_j d_TV; block efficiency: N_acc / N_max
+                    const double r = p.reward_kind == METASD_REWARD_BE ? (double)n_acc / (double)k : sum_align / (double)k;
+                    if (p.diag && lane < k) {
+                        metasd_diag dg;
+                        dg.p_x = r_px;
+                        dg.q_x = r_qx;
+                        dg.D = r_rowflag ? 1.f : (float)(1.0 - smin);
+                        dg.u = h_u;
+                        dg.accept = r_acc;
+                        p.diag[(size_t)b2 * k + lane] = dg;
+                    }
+                    if (lane == 0) {
+                        p.accepted_len[b2] = n_acc;
+                        p.next_token[b2] = drew ? sh.token : token;
+                        p.reward[b2] = (float)r;
+                        if (seq_flags) atomicOr(p.status, seq_flags);
+                    }
+                    warp_bandit(p, b2, h_t, h_arm, r);
+                }
+            }
         }
+        __syncthreads();   // (B) pass 2 is done with its slots
 
-        // ---- end of the sequence: gather sum_v min(p, q) per position in rank 0
-        __syncthreads();
-        if (warp == 0 && lane < k) {
-            double s = 0.0;
-            for (int w = 0; w < nw; ++w) s += (double)sh.pmin[lane][w];
-            st_cluster(map_to_rank(smem_addr(&sh.cta_min[lane][rank]), 0), s);
+        // ---- free and refill pass 2's slots; advance the cursors
+        if (do2) {
+            if (tid == 0) {
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                issue_one();
+                if (pair2) issue_one();
+            }
+            c2 += pair2 ? 2 : 1;
+            if (c2 >= g.n_slot) c2 -= g.n_slot;
+            if (++u2 == 3) { u2 = 0; x2par ^= 1u; }
+            if (++j2 > k) { j2 = 0; b2 += ncl; }
         }
-        cluster_sync_all();
-        if (rank == 0 && warp == 0) {
-            double smin = 0.0;
-            uint32_t rf = 0;
-            if (lane < k) {
-                for (int r = 0; r < csize; ++r) smin += sh.cta_min[lane][r];
-                rf = sh.r_rowflag[lane];
-                if (rf) smin = 0.0;
-            }
-            double sum_align = 0.0;
-            for (int j = 0; j < k; ++j) sum_align += __shfl_sync(0xFFFFFFFFu, smin, j);
-            // Definition 2: 1 - mean_j d_TV; block efficiency: N_acc / N_max
-            const double r = p.reward_kind == METASD_REWARD_BE ? (double)n_acc / (double)k : sum_align / (double)k;
-            if (p.diag && lane < k) {
-                metasd_diag dg;
-                dg.p_x = sh.r_px[lane];
-                dg.q_x = sh.r_qx[lane];
-                dg.D = rf ? 1.f : (float)(1.0 - smin);
-                dg.u = sh.h_u[lane];
-                dg.accept = sh.r_acc[lane];
-                p.diag[(size_t)b * k + lane] = dg;
-            }
-            if (lane == 0) {
-                p.accepted_len[b] = n_acc;
-                p.next_token[b] = drew ? sh.token : token;
-                p.reward[b] = (float)r;
-                if (seq_flags) atomicOr(p.status, seq_flags);
-            }
-            warp_bandit(p, b, sh.h_t, sh.h_arm, r);
+        if (do1) {
+            c1 += pair1 ? 2 : 1;
+            if (c1 >= g.n_slot) { c1 -= g.n_slot; c1par ^= 1u; }
+            if (++u1 == 3) u1 = 0;
+            if (++j1 > k) j1 = 0;
         }
     }
 
-    // ---- no CTA leaves while a copy into its shared memory may be in flight or a peer may still write to it
-    if (tid == 0) {
-        while (consumed < ld_issued) {
-            wait_bar(sh, &sh.full[cs], cpar, p.status);
-            if (++cs == g.n_slot) { cs = 0; cpar ^= 1u; }
-            ++consumed;
-        }
+    // ---- No CTA leaves while a copy into its shared memory may be in flight or a peer may still write to it.
+    // Pass 1 has waited for every copy that was issued, unless a wait ran out: then give the copies one more
+    // bounded delay before the shared memory is given up.
+    if (tid == 0 && *(volatile int32_t *)&sh.dead) {
+        for (uint32_t it = 0; it < (1u << 18); ++it) __nanosleep(256);
     }
     cluster_sync_all();
 }
@@ -816,15 +866,11 @@ __global__ void __launch_bounds__(FUSED_MAX_THREADS, 1) fused_round_kernel(const
 // ---------------------------------------------------------------------------------------------
 // Host side: geometry, occupancy, launch
 // ---------------------------------------------------------------------------------------------
-template <typename LT, int VPT>
-const void *kernel_ptr() { return reinterpret_cast<const void *>(&fused_round_kernel<LT, VPT>); }
-
 const void *kernel_for(int dtype)
 {
-    return dtype == METASD_BF16 ? kernel_ptr<__nv_bfloat16, 5>() : kernel_ptr<float, 10>();
+    return dtype == METASD_BF16 ? reinterpret_cast<const void *>(&fused_round_kernel<__nv_bfloat16>)
+                                : reinterpret_cast<const void *>(&fused_round_kernel<float>);
 }
-
-int vectors_per_thread_max(int dtype) { return dtype == METASD_BF16 ? 5 : 10; }
 
 // Geometry for cluster size C, or false when the row does not fit.
 bool geometry(int dtype, int V, int C, int smem_optin, FusedPlan *pl)
@@ -835,30 +881,26 @@ bool geometry(int dtype, int V, int C, int smem_optin, FusedPlan *pl)
     if (C > n_vec_row) return false;
     const int n_vec_cta = (n_vec_row + C - 1) / C;
     if ((size_t)(C - 1) * n_vec_cta >= (size_t)n_vec_row) return false;   // an empty last rank: a smaller C serves better
-    const int vpt_max = vectors_per_thread_max(dtype);
-    if (n_vec_cta > FUSED_MAX_THREADS * vpt_max) return false;
-    // threads: the multiple of 32 with the least padding, the larger one on ties
-    int best_t = 0;
-    long best_cost = 0;
-    for (int t = FUSED_MAX_THREADS; t >= 64; t -= 32) {
-        const int vpt = (n_vec_cta + t - 1) / t;
-        if (vpt > vpt_max) break;
-        const long cost = (long)t * vpt;
-        if (!best_t || cost < best_cost) { best_t = t; best_cost = cost; }
-    }
-    if (!best_t) return false;
     const int slot_bytes = n_vec_cta * 16;
     int n_slot = (smem_optin - FUSED_SMEM_RESERVE) / slot_bytes;
     if (n_slot > FUSED_MAX_SLOTS) n_slot = FUSED_MAX_SLOTS;
-    if (n_slot < 3) return false;
+    if (n_slot < FUSED_MIN_SLOTS) return false;
+    // streaming warps: the count that divides the slice with the least padding (the larger count on ties),
+    // plus the control warp
+    int best_w = 0;
+    long best_cost = 0;
+    for (int w = FUSED_MAX_WARPS - 1; w >= 1; --w) {
+        const long cost = (long)(w * 32) * ((n_vec_cta + w * 32 - 1) / (w * 32));
+        if (!best_w || cost < best_cost) { best_w = w; best_cost = cost; }
+    }
     pl->cluster = C;
-    pl->threads = best_t;
+    pl->threads = (best_w + 1) * 32;
     pl->n_vec_row = n_vec_row;
     pl->n_vec_cta = n_vec_cta;
     pl->n_slot = n_slot;
     pl->slot_bytes = slot_bytes;
     pl->smem_bytes = (size_t)n_slot * slot_bytes;
-    pl->work_per_item = best_cost;
+    pl->work_per_item = n_vec_cta;
     pl->max_clusters = 0;
     return true;
 }
@@ -900,11 +942,7 @@ cudaError_t fused_prepare(int device, int dtype, int V, int max_batch, FusedPlan
         if (pin_c && C != pin_c) continue;
         FusedPlan pl;
         if (!geometry(dtype, V, C, smem_optin, &pl)) continue;
-        if (pin_t >= 64 && pin_t <= FUSED_MAX_THREADS && pin_t % 32 == 0 &&
-            (pl.n_vec_cta + pin_t - 1) / pin_t <= vectors_per_thread_max(dtype)) {
-            pl.threads = pin_t;
-            pl.work_per_item = (long)pin_t * ((pl.n_vec_cta + pin_t - 1) / pin_t);
-        }
+        if (pin_t >= 64 && pin_t <= FUSED_MAX_THREADS && pin_t % 32 == 0) pl.threads = pin_t;
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(C);
         cfg.blockDim = dim3(pl.threads);
@@ -922,8 +960,8 @@ cudaError_t fused_prepare(int device, int dtype, int V, int max_batch, FusedPlan
         pl.max_clusters = n;
         const int used = n < max_batch ? n : max_batch;
         const double waves = (double)((max_batch + used - 1) / used);
-        // per item: the arithmetic of the slice plus a fixed cost for its barriers and exchanges
-        const double cost = waves * ((double)pl.work_per_item + 400.0);
+        // per item: the two passes over the slice plus a fixed cost for barriers and exchanges
+        const double cost = waves * ((double)pl.work_per_item + 300.0);
         if (!plan->cluster || cost < best) { *plan = pl; best = cost; }
     }
     if (plan->cluster && env_int("METASD_FUSED_VERBOSE", 0))
@@ -952,9 +990,9 @@ cudaError_t launch_fused(const VerifyParams &p, int dtype, const FusedPlan &plan
     cfg.numAttrs = 1;
     cudaError_t e;
     if (dtype == METASD_BF16)
-        e = cudaLaunchKernelEx(&cfg, fused_round_kernel<__nv_bfloat16, 5>, p, g);
+        e = cudaLaunchKernelEx(&cfg, fused_round_kernel<__nv_bfloat16>, p, g);
     else
-        e = cudaLaunchKernelEx(&cfg, fused_round_kernel<float, 10>, p, g);
+        e = cudaLaunchKernelEx(&cfg, fused_round_kernel<float>, p, g);
     *launches += 1;
     return e;
 }
