@@ -169,9 +169,12 @@ struct RowConst {
 struct FusedShared {
     uint64_t full[FUSED_MAX_SLOTS];                      // one mbarrier per ring slot
     uint64_t xbar[3];                                    // arrival of the peers' records, by item mod 3
+    uint64_t wbar[2];                                    // the streaming warps' records are written, by step parity
+    uint64_t rcbar[2];                                   // pass 2's row constants are written, by item parity
+    uint64_t ebar[2];                                    // the streaming warps are done with pass 2's slots, by item parity
     Exchange exch[3][FUSED_MAX_CLUSTER];                 // [item mod 3][sender rank]
-    Exchange wrec[FUSED_MAX_WARPS];                      // the streaming warps' records of the item in pass 1
-    RowConst rc;
+    Exchange wrec[2][FUSED_MAX_WARPS];                   // the streaming warps' records of the item in pass 1
+    RowConst rc[2];
     double tot[FUSED_MAX_WARPS];                         // draw: weight of each streaming warp's range
     double pre[FUSED_MAX_WARPS];                         // draw: exclusive prefix of tot
     double cta_tot[FUSED_MAX_CLUSTER];                   // draw: weight of each CTA's slice
@@ -204,20 +207,6 @@ __device__ __forceinline__ void wait_bar(FusedShared &sh, uint64_t *bar, uint32_
     atomicOr(status, METASD_STATUS_TIMEOUT);
 }
 
-// 16 bytes of logits as pairs of floats.
-template <typename LT>
-__device__ __forceinline__ void unpack2(const uint4 &raw, float2 (&x)[Logit<LT>::VEC / 2])
-{
-    if constexpr (sizeof(LT) == 2) {
-        const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
-#pragma unroll
-        for (int n = 0; n < 4; ++n) x[n] = make_float2(__uint_as_float(w[n] << 16), __uint_as_float(w[n] & 0xFFFF0000u));
-    } else {
-        x[0] = make_float2(__uint_as_float(raw.x), __uint_as_float(raw.y));
-        x[1] = make_float2(__uint_as_float(raw.z), __uint_as_float(raw.w));
-    }
-}
-
 // Largest of the 16 bytes of logits (NaN entries are ignored).
 template <typename LT>
 __device__ __forceinline__ float vector_max(const uint4 &raw)
@@ -231,41 +220,65 @@ __device__ __forceinline__ float vector_max(const uint4 &raw)
     }
 }
 
-// Pass 1 over one row slice in shared memory: the thread's running maximum m, s = sum 2^((x - m) c) and
-// the first vector that set the maximum.  Thread ct of ncomp takes vectors ct, ct + ncomp, ...
-template <typename LT>
-__device__ __forceinline__ void stats_row(const unsigned char *slot, int my_vecs, int ct, int ncomp, float c, float &m_t,
-                                          float &s_t, int &v_t)
+// Pass 1 over one item's row slices in shared memory, by one warp: running maxima shared by the whole
+// warp (so that the rare rescaling branch never diverges), sums 2^((x - max) c) per lane, and per lane the
+// vector in which it first met the target row's maximum.  Thread ct of ncomp takes vectors ct, ct + ncomp, ...;
+// every lane makes the same number of trips, a vector beyond the slice reads as -inf.
+template <typename LT, bool PAIR>
+__device__ __forceinline__ void stats_rows(const unsigned char *slot_a, const unsigned char *slot_b, int my_vecs, int ct,
+                                           int ncomp, int trips, float c, bool want_argmax, float &max_a, float &sum_a,
+                                           int &vec_a, float &max_b, float &sum_b)
 {
-    constexpr int NP = Logit<LT>::VEC / 2;
-    float m = METASD_NEG_BIG;
-    float2 s2 = make_float2(0.f, 0.f);
+    constexpr int VEC = Logit<LT>::VEC;
+    const uint32_t ninf = sizeof(LT) == 2 ? 0xFF80FF80u : 0xFF800000u;
+    float ma = METASD_NEG_BIG, mb = METASD_NEG_BIG;
+    float sa0 = 0.f, sa1 = 0.f, sb0 = 0.f, sb1 = 0.f;
     int bv = -1;
-    const float2 cc = make_float2(c, c);
-#pragma unroll 2
-    for (int v = ct; v < my_vecs; v += ncomp) {
-        const uint4 raw = *reinterpret_cast<const uint4 *>(slot + (size_t)v * 16);
-        const float vm = vector_max<LT>(raw);
-        if (vm > m) {   // rare after the first vectors: rescale the sum to the new maximum
-            const float r = ex2((m - vm) * c);
-            s2.x *= r;
-            s2.y *= r;
-            m = vm;
-            bv = v;
+    for (int i = 0, v = ct; i < trips; ++i, v += ncomp) {
+        uint4 ra = make_uint4(ninf, ninf, ninf, ninf), rb = ra;
+        if (v < my_vecs) {
+            ra = *reinterpret_cast<const uint4 *>(slot_a + (size_t)v * 16);
+            if (PAIR) rb = *reinterpret_cast<const uint4 *>(slot_b + (size_t)v * 16);
         }
-        const float nm = -m * c;
-        const float2 nn = make_float2(nm, nm);
-        float2 x[NP];
-        unpack2<LT>(raw, x);
+        {
+            const float vm = vector_max<LT>(ra);
+            const float wm = warp_max_f(vm);
+            if (wm > ma) {   // warp-uniform, rare after the first vectors: rescale the sums to the new maximum
+                const float r = ex2((ma - wm) * c);
+                sa0 *= r; sa1 *= r;
+                ma = wm;
+                bv = -1;
+            }
+            if (want_argmax && bv < 0 && vm == ma) bv = v;
+            const float nm = -ma * c;
+            float x[VEC];
+            Logit<LT>::unpack(ra, x);
 #pragma unroll
-        for (int n = 0; n < NP; ++n) {
-            const float2 y = __ffma2_rn(x[n], cc, nn);
-            s2 = __fadd2_rn(s2, make_float2(ex2(y.x), ex2(y.y)));
+            for (int q = 0; q < VEC; q += 2) {
+                sa0 += ex2(fmaf(x[q], c, nm));
+                sa1 += ex2(fmaf(x[q + 1], c, nm));
+            }
+        }
+        if (PAIR) {
+            const float vm = vector_max<LT>(rb);
+            const float wm = warp_max_f(vm);
+            if (wm > mb) {
+                const float r = ex2((mb - wm) * c);
+                sb0 *= r; sb1 *= r;
+                mb = wm;
+            }
+            const float nm = -mb * c;
+            float x[VEC];
+            Logit<LT>::unpack(rb, x);
+#pragma unroll
+            for (int q = 0; q < VEC; q += 2) {
+                sb0 += ex2(fmaf(x[q], c, nm));
+                sb1 += ex2(fmaf(x[q + 1], c, nm));
+            }
         }
     }
-    m_t = m;
-    s_t = s2.x + s2.y;
-    v_t = bv;
+    max_a = ma; sum_a = sa0 + sa1; vec_a = bv;
+    max_b = mb; sum_b = sb0 + sb1;
 }
 
 // Pass 2 over one row pair in shared memory: sum_v 2^min(ya_v, yb_v) with ya = x_a c + nma, yb = x_b c + nmb_rel,
@@ -274,23 +287,20 @@ template <typename LT>
 __device__ __forceinline__ float min_rows(const unsigned char *slot_a, const unsigned char *slot_b, int my_vecs, int ct,
                                           int ncomp, float c, float nma, float nmb_rel)
 {
-    constexpr int NP = Logit<LT>::VEC / 2;
-    const float2 cc = make_float2(c, c), na = make_float2(nma, nma), nb = make_float2(nmb_rel, nmb_rel);
-    float2 acc = make_float2(0.f, 0.f);
+    constexpr int VEC = Logit<LT>::VEC;
+    float acc0 = 0.f, acc1 = 0.f;
 #pragma unroll 2
     for (int v = ct; v < my_vecs; v += ncomp) {
-        const uint4 ra = *reinterpret_cast<const uint4 *>(slot_a + (size_t)v * 16);
-        const uint4 rb = *reinterpret_cast<const uint4 *>(slot_b + (size_t)v * 16);
-        float2 xa[NP], xb[NP];
-        unpack2<LT>(ra, xa);
-        unpack2<LT>(rb, xb);
+        float xa[VEC], xb[VEC];
+        Logit<LT>::unpack(*reinterpret_cast<const uint4 *>(slot_a + (size_t)v * 16), xa);
+        Logit<LT>::unpack(*reinterpret_cast<const uint4 *>(slot_b + (size_t)v * 16), xb);
 #pragma unroll
-        for (int n = 0; n < NP; ++n) {
-            const float2 ya = __ffma2_rn(xa[n], cc, na), yb = __ffma2_rn(xb[n], cc, nb);
-            acc = __fadd2_rn(acc, make_float2(ex2(fminf(ya.x, yb.x)), ex2(fminf(ya.y, yb.y))));
+        for (int q = 0; q < VEC; q += 2) {
+            acc0 += ex2(fminf(fmaf(xa[q], c, nma), fmaf(xb[q], c, nmb_rel)));
+            acc1 += ex2(fminf(fmaf(xa[q + 1], c, nma), fmaf(xb[q + 1], c, nmb_rel)));
         }
     }
-    return acc.x + acc.y;
+    return acc0 + acc1;
 }
 
 // Weights of the draw for one vector: mode 1 = max(0, p - q) (correction), mode 2 = p (bonus).
@@ -319,12 +329,11 @@ __device__ __forceinline__ void draw_weights(const unsigned char *slot_a, const 
 // of its CTA's slice; totals and offsets are carried in fp64.  Returns false (for every thread of the
 // cluster alike) when the row has no mass; otherwise the token lands in sh.token of rank 0.
 template <typename LT>
-__device__ bool cluster_draw(FusedShared &sh, const unsigned char *slot_a, const unsigned char *slot_b, int mode, float c,
-                             int my_vecs, int vec0, int rank, int csize, int ncw)
+__device__ bool cluster_draw(FusedShared &sh, const RowConst &rc, const unsigned char *slot_a, const unsigned char *slot_b,
+                             int mode, float c, int my_vecs, int vec0, int rank, int csize, int ncw)
 {
     constexpr int VEC = Logit<LT>::VEC;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const RowConst rc = sh.rc;
     const int per_warp = (my_vecs + ncw - 1) / ncw;
     const int cw = warp - 1;   // streaming warp index; the control warp has none
     const int v0 = cw >= 0 ? min(cw * per_warp, my_vecs) : 0, v1 = cw >= 0 ? min(v0 + per_warp, my_vecs) : 0;
@@ -551,6 +560,11 @@ __global__ void __launch_bounds__(FUSED_MAX_THREADS, 1) fused_round_kernel(const
     if (tid == 0) {
         for (int s = 0; s < g.n_slot; ++s) mbar_init(&sh.full[s], 1);
         for (int s = 0; s < 3; ++s) mbar_init(&sh.xbar[s], 1);
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(&sh.wbar[s], (uint32_t)ncw);
+            mbar_init(&sh.rcbar[s], 1);
+            mbar_init(&sh.ebar[s], (uint32_t)ncw);
+        }
         sh.dead = 0;
         sh.token = -1;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -644,10 +658,16 @@ __global__ void __launch_bounds__(FUSED_MAX_THREADS, 1) fused_round_kernel(const
     uint32_t c1par = 0;
     int u1 = 0, u2 = 0;            // item mod 3 of pass 1 / pass 2: which exchange buffer
     uint32_t x2par = 0;            // phase parity of xbar[u2]
+    const int trips = (my_vecs + ncomp - 1) / ncomp;   // vectors per streaming thread and row slice
 
+    // The streaming warps never meet a CTA-wide barrier in the steady state.  Per step n they hand their
+    // records of item n to the control warp (wbar), pick up the row constants of item n-1 (rcbar) and give
+    // back its slots (ebar); each hand-over is an mbarrier with two buffers, used by alternate steps.
     for (int step = 0; step <= n_items; ++step) {
         const bool do1 = step < n_items, do2 = step >= 1;
         const bool pair1 = j1 < k, pair2 = j2 < k;
+        const int s1 = step & 1, s2 = (step - 1) & 1;                          // buffers of pass 1 / pass 2
+        const uint32_t ph1 = (uint32_t)(step >> 1) & 1u, ph2 = (uint32_t)((step - 1) >> 1) & 1u;   // their phases
         const unsigned char *a2 = ring + (size_t)c2 * g.slot_bytes;
         const unsigned char *d2 = ring + (size_t)(c2 + 1 == g.n_slot ? 0 : c2 + 1) * g.slot_bytes;
 
@@ -728,48 +748,14 @@ __global__ void __launch_bounds__(FUSED_MAX_THREADS, 1) fused_round_kernel(const
                     rc.u_draw = ud;
                     rc.mode = mode;
                     rc.valid = rowflag ? 0 : 1;
-                    sh.rc = rc;
+                    sh.rc[s2] = rc;
+                    mbar_arrive(&sh.rcbar[s2]);   // release: the streaming warps may start pass 2 of this item
                 }
             }
-        } else if (do1) {
-            // ---- pass 1: statistics of this item's row slices out of shared memory
-            Exchange wr;
-            float m_t, s_t;
-            int v_t, v_dummy;
-            const unsigned char *slot = ring + (size_t)c1 * g.slot_bytes;
-            wait_bar(sh, &sh.full[c1], c1par, p.status);
-            stats_row<LT>(slot, my_vecs, ct, ncomp, c, m_t, s_t, v_t);
-            wr.max_a = warp_max_f(m_t);
-            wr.sum_a = warp_sum_f(s_t * ex2((m_t - wr.max_a) * c));
-            int cand = INT_MAX;
-            if (p.greedy && m_t == wr.max_a && v_t >= 0) {   // first index of the maximum inside the vector that set it
-                float x[VEC];
-                Logit<LT>::unpack(*reinterpret_cast<const uint4 *>(slot + (size_t)v_t * 16), x);
-#pragma unroll
-                for (int q = VEC - 1; q >= 0; --q)
-                    if (x[q] == m_t) cand = (vec0 + v_t) * VEC + q;
-            }
-            wr.idx_a = p.greedy ? __reduce_min_sync(0xFFFFFFFFu, cand) : INT_MAX;
-            wr.max_b = METASD_NEG_BIG;
-            wr.sum_b = 0.f;
-            if (pair1) {
-                const int cb = c1 + 1 == g.n_slot ? 0 : c1 + 1;
-                wait_bar(sh, &sh.full[cb], cb == 0 ? c1par ^ 1u : c1par, p.status);
-                stats_row<LT>(ring + (size_t)cb * g.slot_bytes, my_vecs, ct, ncomp, c, m_t, s_t, v_dummy);
-                wr.max_b = warp_max_f(m_t);
-                wr.sum_b = warp_sum_f(s_t * ex2((m_t - wr.max_b) * c));
-            }
-            if (lane == 0) {
-                wr.pad[0] = wr.pad[1] = wr.pad[2] = 0;
-                sh.wrec[warp - 1] = wr;
-            }
-        }
-        __syncthreads();   // (C) the warps' records and pass 2's row constants are in shared memory
-
-        if (control) {
             // ---- the CTA's record of pass 1's item goes to every CTA of the cluster
             if (do1) {
-                const Merged mc = merge_records(sh.wrec, ncw, lane, c);
+                wait_bar(sh, &sh.wbar[s1], ph1, p.status);
+                const Merged mc = merge_records(sh.wrec[s1], ncw, lane, c);
                 if (lane < csize) {
                     const uint32_t dst = map_to_rank(smem_addr(&sh.exch[u1][rank]), (uint32_t)lane);
                     const uint32_t bar = map_to_rank(smem_addr(&sh.xbar[u1]), (uint32_t)lane);
@@ -778,20 +764,57 @@ __global__ void __launch_bounds__(FUSED_MAX_THREADS, 1) fused_round_kernel(const
                     st_async_16(dst + 16, bar, (uint32_t)mc.idx, 0u, 0u, 0u);
                 }
             }
-        } else if (do2 && pair2) {
-            // ---- pass 2: sum_v min(p_v, q_v) of this warp's logits
-            const RowConst rc = sh.rc;
-            float acc = 0.f;
-            if (rc.valid) acc = min_rows<LT>(a2, d2, my_vecs, ct, ncomp, c, rc.nma, rc.nmb_rel) * rc.inv_sa;
-            acc = warp_sum_f(acc);
-            if (lane == 0) sh.pmin[j2][warp - 1] = acc;
+        } else {
+            if (do1) {
+                // ---- pass 1: statistics of this item's row slices out of shared memory
+                Exchange wr;
+                int v_t;
+                const int cb = c1 + 1 == g.n_slot ? 0 : c1 + 1;
+                const unsigned char *slot_a = ring + (size_t)c1 * g.slot_bytes, *slot_b = ring + (size_t)cb * g.slot_bytes;
+                wait_bar(sh, &sh.full[c1], c1par, p.status);
+                if (pair1) {
+                    wait_bar(sh, &sh.full[cb], cb == 0 ? c1par ^ 1u : c1par, p.status);
+                    stats_rows<LT, true>(slot_a, slot_b, my_vecs, ct, ncomp, trips, c, p.greedy != 0, wr.max_a, wr.sum_a, v_t,
+                                         wr.max_b, wr.sum_b);
+                } else {
+                    stats_rows<LT, false>(slot_a, slot_b, my_vecs, ct, ncomp, trips, c, p.greedy != 0, wr.max_a, wr.sum_a, v_t,
+                                          wr.max_b, wr.sum_b);
+                }
+                int cand = INT_MAX;
+                if (v_t >= 0) {   // first index of the maximum inside the vector in which this lane met it
+                    float x[VEC];
+                    Logit<LT>::unpack(*reinterpret_cast<const uint4 *>(slot_a + (size_t)v_t * 16), x);
+#pragma unroll
+                    for (int q = VEC - 1; q >= 0; --q)
+                        if (x[q] == wr.max_a) cand = (vec0 + v_t) * VEC + q;
+                }
+                wr.idx_a = p.greedy ? __reduce_min_sync(0xFFFFFFFFu, cand) : INT_MAX;
+                wr.sum_a = warp_sum_f(wr.sum_a);   // the lanes share one maximum per row
+                wr.sum_b = warp_sum_f(wr.sum_b);
+                if (lane == 0) {
+                    wr.pad[0] = wr.pad[1] = wr.pad[2] = 0;
+                    sh.wrec[s1][warp - 1] = wr;
+                    mbar_arrive(&sh.wbar[s1]);
+                }
+            }
+            if (do2) {
+                // ---- pass 2: sum_v min(p_v, q_v) of this warp's logits
+                wait_bar(sh, &sh.rcbar[s2], ph2, p.status);
+                if (pair2) {
+                    const RowConst rc = sh.rc[s2];
+                    float acc = 0.f;
+                    if (rc.valid) acc = min_rows<LT>(a2, d2, my_vecs, ct, ncomp, c, rc.nma, rc.nmb_rel) * rc.inv_sa;
+                    acc = warp_sum_f(acc);
+                    if (lane == 0) sh.pmin[j2][warp - 1] = acc;
+                }
+            }
         }
         if (do2) {
-            const int mode = sh.rc.mode;   // alike in every thread of the cluster
+            const int mode = sh.rc[s2].mode;   // alike in every thread of the cluster; the control warp wrote it
             if (mode) {
-                bool ok = cluster_draw<LT>(sh, a2, d2, mode, c, my_vecs, vec0, rank, csize, ncw);
+                bool ok = cluster_draw<LT>(sh, sh.rc[s2], a2, d2, mode, c, my_vecs, vec0, rank, csize, ncw);
                 if (!ok && mode == 1)   // p == q in fp32 yet rejected: draw from p
-                    ok = cluster_draw<LT>(sh, a2, d2, 2, c, my_vecs, vec0, rank, csize, ncw);
+                    ok = cluster_draw<LT>(sh, sh.rc[s2], a2, d2, 2, c, my_vecs, vec0, rank, csize, ncw);
                 drew = ok;
             }
             if (!pair2) {
@@ -831,15 +854,18 @@ __global__ void __launch_bounds__(FUSED_MAX_THREADS, 1) fused_round_kernel(const
                     warp_bandit(p, b2, h_t, h_arm, r);
                 }
             }
-        }
-        __syncthreads();   // (B) pass 2 is done with its slots
-
-        // ---- free and refill pass 2's slots; advance the cursors
-        if (do2) {
-            if (tid == 0) {
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                issue_one();
-                if (pair2) issue_one();
+            // ---- pass 2's slots go back to the ring: the streaming warps sign off, the control warp refills
+            if (!control) {
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sh.ebar[s2]);
+            } else {
+                wait_bar(sh, &sh.ebar[s2], ph2, p.status);
+                if (lane == 0) {
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    issue_one();
+                    if (pair2) issue_one();
+                }
+                __syncwarp();
             }
             c2 += pair2 ? 2 : 1;
             if (c2 >= g.n_slot) c2 -= g.n_slot;
