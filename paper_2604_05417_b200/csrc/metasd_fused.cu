@@ -1,26 +1,22 @@
 // Fused cluster path of the MetaSD verify round: ONE persistent kernel per call.
 //
 // A thread-block cluster of C CTAs owns one sequence at a time and walks its k+1 positions in order.
-// Every CTA owns a contiguous 1/C slice of each logit row.  The slices arrive in shared memory through
-// a ring of bulk asynchronous copies (TMA, completion on an mbarrier) that runs ahead of the arithmetic,
-// so each logit is read from HBM exactly once and stays on chip for both passes over it:
-//
-//   pass 1 (row statistics)  per row: running maximum and sum_v 2^((x_v - max) c); the CTA's record
-//                            (max, sum, first arg-max) goes to every CTA of the cluster as asynchronous
-//                            distributed-shared-memory stores that complete on the receiver's mbarrier;
-//   pass 2 (one item later)  with the merged records of the whole row pair:
-//                              sum_v min(p_v, q_v) = 1 - d_TV(p_j, q_j)            (Definition 2, Eq. 4)
-//                            evaluated as sum_v 2^min(log2 p_v, log2 q_v): one exponential per PAIR;
-//                            the accept test u q(x) < p(x) of the drafted token     (Algorithm 4, l. 7-8);
-//                            at the first rejection (or the bonus position) the inverse-CDF draw from
-//                            max(0, p - q) (or p), a prefix search in token order across the cluster
-//                                                                                    (Algorithm 4, l. 11-12).
-//
-// Pass 2 of item n-1 runs after pass 1 of item n, so the latency of the record exchange hides behind a
-// full pass.  Warp 0 of every CTA is a control warp (lane j = position j of the sequence): it issues the
-// copies, merges and sends records, runs the accept tests, and in rank 0 writes the outputs, forms the
-// reward and updates the bandit with one lane per drafter (Algorithm 2, lines 7-10).  The other warps
-// only stream logits out of shared memory.
+// Every CTA owns a contiguous 1/C slice of each logit row; C is the smallest size for which a slice
+// pair (target + draft) fits half an SM's shared memory, so that TWO CTAs (of different clusters) live
+// on every SM and fill each other's waits.  Per position a CTA
+//   - receives its two slices through bulk asynchronous copies (TMA), a few chunks per slice, each
+//     completing on its own mbarrier: every logit is read from HBM exactly once;
+//   - pass 1, chunk by chunk as they land: running maximum and sum_v 2^((x_v - max) c) of both rows, the
+//     first arg-max of the target row; the CTA's record goes to every CTA of the cluster as asynchronous
+//     distributed-shared-memory stores that complete on the receiver's mbarrier;
+//   - pass 2, over the same bytes still in shared memory, with the merged records of the whole row pair:
+//       sum_v min(p_v, q_v) = 1 - d_TV(p_j, q_j)  (Definition 2, Eq. 4), evaluated as
+//       sum_v 2^min(log2 p_v, log2 q_v): one exponential per PAIR;
+//     the accept test u q(x) < p(x) of the drafted token (Algorithm 4, lines 7-8), evaluated alike by
+//     every thread of the cluster; at the first rejection (or the bonus position) the inverse-CDF draw
+//     from max(0, p - q) (or p), a prefix search in token order across the cluster (Algorithm 4, 11-12).
+// Rank 0 of the cluster then writes the outputs, forms the reward, and one warp updates the bandit and
+// selects the next arm with one lane per drafter (Algorithm 2, lines 7-10).
 #include <limits.h>
 #include <stdio.h>
 #include <stdlib.h>
@@ -31,12 +27,11 @@ namespace metasd {
 
 namespace {
 
-constexpr int FUSED_MAX_THREADS = 1024;
-constexpr int FUSED_MAX_WARPS = FUSED_MAX_THREADS / 32;
+constexpr int FUSED_MAX_THREADS = 640;            // two CTAs per SM: 1280 threads, about 50 registers each
+constexpr int FUSED_MAX_WARPS = 32;
 constexpr int FUSED_MAX_CLUSTER = 16;
-constexpr int FUSED_MAX_SLOTS = 8;
-constexpr int FUSED_MIN_SLOTS = 5;                // two items of two rows each, plus one copy in flight
-constexpr int FUSED_SMEM_RESERVE = 12 * 1024;     // static shared memory + slack kept out of the ring
+constexpr int FUSED_CHUNKS = 4;                   // bulk copies (and mbarriers) per row slice
+constexpr int FUSED_STATIC_SMEM = 9 * 1024;       // static shared memory of one CTA, rounded up
 constexpr uint32_t WAIT_FAST_POLLS = 4096u;
 constexpr uint32_t WAIT_SLOW_POLLS = 1u << 21;    // with a back-off of 128 ns each: a few tenths of a second
 
@@ -156,40 +151,42 @@ struct __align__(16) Exchange {   // (max, sum) of both rows and the first arg-m
 };
 constexpr uint32_t EXCHANGE_BYTES = 32;
 
-// What the control warp hands to the streaming warps for pass 2 of one item.
+// Constants of one row pair, known once the cluster's records are merged.
 struct RowConst {
     float nma, nmb;      // -max c of the target / draft row
     float nmb_rel;       // nmb + log2(sum_a / sum_b): the draft row on the target row's scale
     float inv_sa, inv_sb;
     float u_draw;        // uniform of the residual / bonus draw
-    int32_t mode;        // 0 none, 1 draw from max(0, p - q), 2 draw from p
-    int32_t valid;       // 0: the row pair is flagged non-finite, its sum of minima is 0
 };
 
 struct FusedShared {
-    uint64_t full[FUSED_MAX_SLOTS];                      // one mbarrier per ring slot
-    uint64_t xbar[3];                                    // arrival of the peers' records, by item mod 3
-    uint64_t wbar[2];                                    // the streaming warps' records are written, by step parity
-    uint64_t rcbar[2];                                   // pass 2's row constants are written, by item parity
-    uint64_t ebar[2];                                    // the streaming warps are done with pass 2's slots, by item parity
-    Exchange exch[3][FUSED_MAX_CLUSTER];                 // [item mod 3][sender rank]
-    Exchange wrec[2][FUSED_MAX_WARPS];                   // the streaming warps' records of the item in pass 1
-    RowConst rc[2];
-    double tot[FUSED_MAX_WARPS];                         // draw: weight of each streaming warp's range
+    uint64_t full[2][FUSED_CHUNKS];                      // [row][chunk]: the chunk's bytes have landed
+    uint64_t xbar[2];                                    // arrival of the peers' records, by item parity
+    Exchange exch[2][FUSED_MAX_CLUSTER];                 // [item parity][sender rank]
+    Exchange wrec[FUSED_MAX_WARPS];                      // the warps' records of the item
+    double tot[FUSED_MAX_WARPS];                         // draw: weight of each warp's range
     double pre[FUSED_MAX_WARPS];                         // draw: exclusive prefix of tot
     double cta_tot[FUSED_MAX_CLUSTER];                   // draw: weight of each CTA's slice
     double cta_min[16][FUSED_MAX_CLUSTER];               // rank 0: sum of min(p, q) per position and sender
-    float pmin[16][FUSED_MAX_WARPS];                     // sum of min(p, q) per position and streaming warp
+    float pmin[16][FUSED_MAX_WARPS];                     // sum of min(p, q) per position and warp
     const void *table[16];                               // the drafter pointer table
+    // header of the current sequence
+    int32_t h_tok[16];
+    float h_xa[16], h_xb[16], h_u[16], h_ud[17];
+    int32_t h_t, h_arm;
+    // per-position results of the current sequence
+    int32_t r_acc[16];
+    float r_px[16], r_qx[16];
+    uint32_t r_rowflag[16];
     int32_t token;                                       // rank 0: the drawn token
     int32_t dead;                                        // a wait ran out: later waits do not spin again
 };
 
 struct FusedGeom {
-    int32_t n_vec_row;   // 16-byte vectors per logit row
-    int32_t n_vec_cta;   // vectors of a row owned by one CTA (the last ranks may own fewer)
-    int32_t n_slot;      // ring slots
-    int32_t slot_bytes;  // n_vec_cta * 16
+    int32_t n_vec_row;    // 16-byte vectors per logit row
+    int32_t n_vec_cta;    // vectors of a row owned by one CTA (the last ranks may own fewer)
+    int32_t slot_bytes;   // n_vec_cta * 16
+    int32_t chunk_shift;  // a chunk is 1 << chunk_shift vectors
 };
 
 // Waits for a phase of an mbarrier.  Bounded: after the limit the CTA is marked dead, the status word
@@ -222,21 +219,29 @@ __device__ __forceinline__ float vector_max(const uint4 &raw)
 
 // Pass 1 over one item's row slices in shared memory, by one warp: running maxima shared by the whole
 // warp (so that the rare rescaling branch never diverges), sums 2^((x - max) c) per lane, and per lane the
-// vector in which it first met the target row's maximum.  Thread ct of ncomp takes vectors ct, ct + ncomp, ...;
-// every lane makes the same number of trips, a vector beyond the slice reads as -inf.
+// vector in which it first met the target row's maximum.  Thread ct of nthr takes vectors ct, ct + nthr, ...;
+// every lane makes the same number of trips, a vector beyond the slice reads as -inf.  A lane waits for the
+// chunk that holds its vector before it reads it.
 template <typename LT, bool PAIR>
-__device__ __forceinline__ void stats_rows(const unsigned char *slot_a, const unsigned char *slot_b, int my_vecs, int ct,
-                                           int ncomp, int trips, float c, bool want_argmax, float &max_a, float &sum_a,
+__device__ __forceinline__ void stats_rows(FusedShared &sh, uint32_t *status, const unsigned char *slot_a,
+                                           const unsigned char *slot_b, uint32_t par_a, uint32_t par_b, int chunk_shift,
+                                           int my_vecs, int ct, int nthr, int trips, float c, float &max_a, float &sum_a,
                                            int &vec_a, float &max_b, float &sum_b)
 {
     constexpr int VEC = Logit<LT>::VEC;
     const uint32_t ninf = sizeof(LT) == 2 ? 0xFF80FF80u : 0xFF800000u;
     float ma = METASD_NEG_BIG, mb = METASD_NEG_BIG;
     float sa0 = 0.f, sa1 = 0.f, sb0 = 0.f, sb1 = 0.f;
-    int bv = -1;
-    for (int i = 0, v = ct; i < trips; ++i, v += ncomp) {
+    int bv = -1, ready = 0;   // chunks [0, ready) of both rows are known to have landed
+    for (int i = 0, v = ct; i < trips; ++i, v += nthr) {
         uint4 ra = make_uint4(ninf, ninf, ninf, ninf), rb = ra;
         if (v < my_vecs) {
+            const int need = v >> chunk_shift;
+            while (ready <= need) {
+                wait_bar(sh, &sh.full[0][ready], par_a, status);
+                if (PAIR) wait_bar(sh, &sh.full[1][ready], par_b, status);
+                ++ready;
+            }
             ra = *reinterpret_cast<const uint4 *>(slot_a + (size_t)v * 16);
             if (PAIR) rb = *reinterpret_cast<const uint4 *>(slot_b + (size_t)v * 16);
         }
@@ -249,7 +254,7 @@ __device__ __forceinline__ void stats_rows(const unsigned char *slot_a, const un
                 ma = wm;
                 bv = -1;
             }
-            if (want_argmax && bv < 0 && vm == ma) bv = v;
+            if (bv < 0 && vm == ma) bv = v;
             const float nm = -ma * c;
             float x[VEC];
             Logit<LT>::unpack(ra, x);
@@ -325,8 +330,8 @@ __device__ __forceinline__ void draw_weights(const unsigned char *slot_a, const 
 }
 
 // Inverse CDF in token order over one row (pair) that lives in the shared memory of the whole cluster:
-// the smallest v with sum_{w <= v} weight_w > u * total.  Every streaming warp owns a contiguous range
-// of its CTA's slice; totals and offsets are carried in fp64.  Returns false (for every thread of the
+// the smallest v with sum_{w <= v} weight_w > u * total.  Every warp owns a contiguous range of its
+// CTA's slice; totals and offsets are carried in fp64.  Returns false (for every thread of the
 // cluster alike) when the row has no mass; otherwise the token lands in sh.token of rank 0.
 template <typename LT>
 __device__ bool cluster_draw(FusedShared &sh, const RowConst &rc, const unsigned char *slot_a, const unsigned char *slot_b,
@@ -335,9 +340,9 @@ __device__ bool cluster_draw(FusedShared &sh, const RowConst &rc, const unsigned
     constexpr int VEC = Logit<LT>::VEC;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int per_warp = (my_vecs + ncw - 1) / ncw;
-    const int cw = warp - 1;   // streaming warp index; the control warp has none
-    const int v0 = cw >= 0 ? min(cw * per_warp, my_vecs) : 0, v1 = cw >= 0 ? min(v0 + per_warp, my_vecs) : 0;
-    if (cw >= 0) {
+    const int cw = warp;
+    const int v0 = min(cw * per_warp, my_vecs), v1 = min(v0 + per_warp, my_vecs);
+    {
         double acc = 0.0;
         for (int v = v0 + lane; v < v1; v += 32) {
             float w[VEC];
@@ -384,7 +389,7 @@ __device__ bool cluster_draw(FusedShared &sh, const RowConst &rc, const unsigned
         }
     }
     if (rstar < 0) rstar = rlast;   // rounding left the total a hair under the threshold
-    if (rank == rstar && cw >= 0) {
+    if (rank == rstar) {
         const double th = thr - mybase;
         // the warp whose range holds the crossing; rounding may leave none: then the last warp with mass
         const double t = lane < ncw ? sh.tot[lane] : 0.0;
@@ -538,16 +543,14 @@ __device__ void warp_bandit(const VerifyParams &p, int b, int t, int arm, double
 // The kernel
 // ---------------------------------------------------------------------------------------------
 template <typename LT>
-__global__ void __launch_bounds__(FUSED_MAX_THREADS, 1) fused_round_kernel(const VerifyParams p, const FusedGeom g)
+__global__ void __launch_bounds__(FUSED_MAX_THREADS, 2) fused_round_kernel(const VerifyParams p, const FusedGeom g)
 {
     constexpr int VEC = Logit<LT>::VEC;
-    extern __shared__ __align__(128) unsigned char ring[];
+    extern __shared__ __align__(128) unsigned char slices[];   // target slice, then draft slice
     __shared__ FusedShared sh;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int ncw = (blockDim.x >> 5) - 1;            // streaming warps
-    const int ncomp = ncw * 32, ct = tid - 32;        // streaming threads and this thread's index among them
-    const bool control = warp == 0;
+    const int nthr = blockDim.x, nw = nthr >> 5;
     const int rank = (int)cluster_rank(), csize = (int)cluster_size();
     const int cid = (int)cluster_id(), ncl = (int)cluster_count();
     const int k = p.k, V = p.V;
@@ -555,16 +558,16 @@ __global__ void __launch_bounds__(FUSED_MAX_THREADS, 1) fused_round_kernel(const
     const size_t row_bytes = (size_t)V * sizeof(LT);
     const int vec0 = rank * g.n_vec_cta;
     const int my_vecs = max(0, min(g.n_vec_cta, g.n_vec_row - vec0));
-    const uint32_t my_bytes = (uint32_t)my_vecs * 16u;
+    const int chunk_vecs = 1 << g.chunk_shift;
+    const int n_chunk = (my_vecs + chunk_vecs - 1) >> g.chunk_shift;
+    const int trips = (my_vecs + nthr - 1) / nthr;   // vectors per thread and row slice
+    unsigned char *slot_a = slices, *slot_b = slices + g.slot_bytes;
 
     if (tid == 0) {
-        for (int s = 0; s < g.n_slot; ++s) mbar_init(&sh.full[s], 1);
-        for (int s = 0; s < 3; ++s) mbar_init(&sh.xbar[s], 1);
-        for (int s = 0; s < 2; ++s) {
-            mbar_init(&sh.wbar[s], (uint32_t)ncw);
-            mbar_init(&sh.rcbar[s], 1);
-            mbar_init(&sh.ebar[s], (uint32_t)ncw);
-        }
+        for (int r = 0; r < 2; ++r)
+            for (int ch = 0; ch < FUSED_CHUNKS; ++ch) mbar_init(&sh.full[r][ch], 1);
+        mbar_init(&sh.xbar[0], 1);
+        mbar_init(&sh.xbar[1], 1);
         sh.dead = 0;
         sh.token = -1;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -572,53 +575,50 @@ __global__ void __launch_bounds__(FUSED_MAX_THREADS, 1) fused_round_kernel(const
     if (tid < 16) sh.table[tid] = (p.drafter_ptrs && tid < p.K) ? p.drafter_ptrs[tid] : nullptr;
     cluster_sync_all();   // every CTA of the cluster is running, its barriers initialised, before a peer writes to it
 
-    const int n_seq = cid < p.batch ? (p.batch - cid + ncl - 1) / ncl : 0;   // sequences of this cluster
-    const int n_items = n_seq * (k + 1);
-
-    // ---- producer (thread 0): the order of loads is sequence-major, position, target then draft
-    int ld_b = cid, ld_j = 0, ld_row = 0, ld_slot = 0, ld_arm_next = 0;
+    // ---- producer (thread 0): one item = the chunks of a target slice and, below the bonus position, of a draft slice
+    int ld_b = cid, ld_j = 0, ld_arm_next = 0;
     const unsigned char *ld_draft = nullptr;
     auto draft_base = [&](int arm) -> const unsigned char * {
         return reinterpret_cast<const unsigned char *>(p.draft ? p.draft : sh.table[arm & 15]);
     };
-    auto issue_one = [&]() {
-        if (ld_b >= p.batch || *(volatile int32_t *)&sh.dead) return;   // after a time-out nothing more is armed
-        const unsigned char *base = ld_row == 0 ? reinterpret_cast<const unsigned char *>(p.target) : ld_draft;
-        const unsigned char *src =
-            base + (ld_row == 0 ? ((size_t)ld_b * (k + 1) + ld_j) : ((size_t)ld_b * k + ld_j)) * row_bytes + (size_t)vec0 * 16;
-        uint64_t *bar = &sh.full[ld_slot];
-        if (my_bytes == 0) {
-            mbar_arrive(bar);
-        } else if (base == nullptr || (reinterpret_cast<uintptr_t>(src) & 15u) != 0) {
-            atomicOr(p.status, METASD_STATUS_BAD_POINTER);   // never hand a misaligned address to the copy engine
-            mbar_arrive(bar);
-        } else {
-            mbar_arrive_expect_tx(bar, my_bytes);
-            bulk_load(ring + (size_t)ld_slot * g.slot_bytes, src, my_bytes, bar);
-        }
-        ld_slot = ld_slot + 1 == g.n_slot ? 0 : ld_slot + 1;
-        if (ld_row == 0 && ld_j < k) {
-            ld_row = 1;
-        } else {
-            ld_row = 0;
-            if (++ld_j > k) {
-                ld_j = 0;
-                ld_b += ncl;
-                if (ld_b < p.batch) {
-                    ld_draft = draft_base(ld_arm_next);
-                    if (!p.draft && ld_b + ncl < p.batch) ld_arm_next = p.st.arm[ld_b + ncl];
-                }
+    auto issue_row = [&](int row, const unsigned char *base, size_t row_index) {
+        const unsigned char *src = base + row_index * row_bytes + (size_t)vec0 * 16;
+        const bool bad = base == nullptr || (reinterpret_cast<uintptr_t>(src) & 15u) != 0;
+        if (bad) atomicOr(p.status, METASD_STATUS_BAD_POINTER);   // never hand a misaligned address to the copy engine
+        unsigned char *dst = row == 0 ? slot_a : slot_b;
+        for (int ch = 0; ch < n_chunk; ++ch) {
+            const int v_lo = ch << g.chunk_shift;
+            const uint32_t bytes = (uint32_t)(min(my_vecs, v_lo + chunk_vecs) - v_lo) * 16u;
+            uint64_t *bar = &sh.full[row][ch];
+            if (bad) {
+                mbar_arrive(bar);
+            } else {
+                mbar_arrive_expect_tx(bar, bytes);
+                bulk_load(dst + (size_t)v_lo * 16, src + (size_t)v_lo * 16, bytes, bar);
             }
         }
     };
-    if (tid == 0 && n_seq > 0) {
+    auto issue_item = [&]() {
+        if (ld_b >= p.batch || *(volatile int32_t *)&sh.dead) return;   // after a time-out nothing more is armed
+        issue_row(0, reinterpret_cast<const unsigned char *>(p.target), (size_t)ld_b * (k + 1) + ld_j);
+        if (ld_j < k) issue_row(1, ld_draft, (size_t)ld_b * k + ld_j);
+        if (++ld_j > k) {
+            ld_j = 0;
+            ld_b += ncl;
+            if (ld_b < p.batch) {
+                ld_draft = draft_base(ld_arm_next);
+                if (!p.draft && ld_b + ncl < p.batch) ld_arm_next = p.st.arm[ld_b + ncl];
+            }
+        }
+    };
+    if (tid == 0 && cid < p.batch) {
         ld_draft = draft_base(p.draft ? 0 : p.st.arm[cid]);
         if (!p.draft && cid + ncl < p.batch) ld_arm_next = p.st.arm[cid + ncl];
-        for (int s = 0; s < g.n_slot; ++s) issue_one();
+        issue_item();
     }
 
-    // ---- control warp, lane j = position j: header of a sequence (round counter, arm, drafted token, its
-    // two logits), fetched one sequence ahead in three steps spread over the items
+    // ---- header of a sequence (warp 0, lane j = position j): round counter, arm, drafted token and
+    // its two logits.  Fetched one sequence ahead, in three steps spread over the items.
     int nx_t = 0, nx_arm = 0, nx_tok = -1;
     float nx_xa = 0.f, nx_xb = 0.f;
     auto fetch_step = [&](int b, int step) {
@@ -641,147 +641,62 @@ __global__ void __launch_bounds__(FUSED_MAX_THREADS, 1) fused_round_kernel(const
             }
         }
     };
-    if (control && n_seq > 0) {
+    if (warp == 0 && cid < p.batch) {
         fetch_step(cid, 0);
         fetch_step(cid, 1);
         fetch_step(cid, 2);
     }
-    // header and results of the sequence in pass 2 (control warp registers, lane j = position j)
-    int h_t = 0, h_arm = 0, h_tok = -1, r_acc = 0;
-    float h_xa = 0.f, h_xb = 0.f, h_u = 0.f, h_ud = 0.f, r_px = 0.f, r_qx = 0.f;
-    uint32_t r_rowflag = 0, seq_flags = 0;
-    int n_acc = -1, token = -1;   // n_acc < 0: no rejection yet
-    bool drew = false;            // the token sits in sh.token of rank 0
 
-    // cursors: pass 1 consumes ring slots c1, pass 2 (one item behind) reads slots c2 and then frees them
-    int j1 = 0, c1 = 0, b2 = cid, j2 = 0, c2 = 0;
-    uint32_t c1par = 0;
-    int u1 = 0, u2 = 0;            // item mod 3 of pass 1 / pass 2: which exchange buffer
-    uint32_t x2par = 0;            // phase parity of xbar[u2]
-    const int trips = (my_vecs + ncomp - 1) / ncomp;   // vectors per streaming thread and row slice
+    uint32_t item = 0;       // items done by this cluster: bit 0 selects the exchange buffers, bit 1 their phase
+    uint32_t par_a = 0, par_b = 0;   // phase parities of the target / draft chunk barriers
 
-    // The streaming warps never meet a CTA-wide barrier in the steady state.  Per step n they hand their
-    // records of item n to the control warp (wbar), pick up the row constants of item n-1 (rcbar) and give
-    // back its slots (ebar); each hand-over is an mbarrier with two buffers, used by alternate steps.
-    for (int step = 0; step <= n_items; ++step) {
-        const bool do1 = step < n_items, do2 = step >= 1;
-        const bool pair1 = j1 < k, pair2 = j2 < k;
-        const int s1 = step & 1, s2 = (step - 1) & 1;                          // buffers of pass 1 / pass 2
-        const uint32_t ph1 = (uint32_t)(step >> 1) & 1u, ph2 = (uint32_t)((step - 1) >> 1) & 1u;   // their phases
-        const unsigned char *a2 = ring + (size_t)c2 * g.slot_bytes;
-        const unsigned char *d2 = ring + (size_t)(c2 + 1 == g.n_slot ? 0 : c2 + 1) * g.slot_bytes;
-
-        if (control) {
-            // ---- expect one record of 32 bytes from every CTA of the cluster (this one included) for pass 1's item
-            if (do1 && lane == 0 && !*(volatile int32_t *)&sh.dead)
-                mbar_arrive_expect_tx(&sh.xbar[u1], (uint32_t)csize * EXCHANGE_BYTES);
-            if (do2) {
-                // ---- pass 2's item: merged records, flags, the accept test of Algorithm 4 (lines 7-8), what to draw
-                if (j2 == 0) {   // a new sequence enters pass 2
-                    h_t = nx_t; h_arm = nx_arm; h_tok = nx_tok; h_xa = nx_xa; h_xb = nx_xb;
-                    const uint4 w = round_words(p.seed, p.sequence_base + (uint32_t)b2, (uint32_t)h_t, (uint32_t)lane);
-                    h_u = uniform24(w.x);
-                    h_ud = uniform24(w.y);
-                    n_acc = -1; token = -1; drew = false; seq_flags = 0; r_acc = 0; r_px = 0.f; r_qx = 0.f; r_rowflag = 0;
+    for (int b = cid; b < p.batch; b += ncl) {
+        // ---- publish the header of sequence b (read after the next CTA barrier)
+        if (warp == 0) {
+            if (lane == 0) { sh.h_t = nx_t; sh.h_arm = nx_arm; }
+            if (lane <= k) {
+                const uint4 w = round_words(p.seed, p.sequence_base + (uint32_t)b, (uint32_t)nx_t, (uint32_t)lane);
+                sh.h_ud[lane] = uniform24(w.y);
+                if (lane < k) {
+                    sh.h_u[lane] = uniform24(w.x);
+                    sh.h_tok[lane] = nx_tok;
+                    sh.h_xa[lane] = nx_xa;
+                    sh.h_xb[lane] = nx_xb;
                 }
-                const int b_next = b2 + ncl;
+            }
+        }
+        const int b_next = b + ncl;
+        int n_acc = -1;          // undecided
+        int token = -1;
+        bool drew = false;       // the token sits in sh.token of rank 0
+        uint32_t seq_flags = 0;
+
+        for (int j = 0; j <= k; ++j, ++item) {
+            const bool pair = j < k;
+            const int par = item & 1;
+            if (warp == 0) {
                 if (b_next < p.batch) {
-                    if (j2 == 0) fetch_step(b_next, 0);
-                    if (j2 == 1) fetch_step(b_next, 1);
-                    if (j2 == (k < 2 ? k : 2)) fetch_step(b_next, 2);
+                    if (j == 0) fetch_step(b_next, 0);
+                    if (j == 1) fetch_step(b_next, 1);
+                    if (j == (k < 2 ? k : 2)) fetch_step(b_next, 2);
                 }
-                wait_bar(sh, &sh.xbar[u2], x2par, p.status);
-                const Merged mg = merge_records(sh.exch[u2], csize, lane, c);
-                // NaN or +Inf anywhere makes the sum NaN; an all -Inf row leaves it 0
-                const bool bad_a = !(mg.Sa > 0.f) || !(mg.Sa < INFINITY) || !(mg.Ma < INFINITY);
-                const bool bad_b = pair2 && (!(mg.Sb > 0.f) || !(mg.Sb < INFINITY) || !(mg.Mb < INFINITY));
-                const uint32_t rowflag = (bad_a || bad_b) ? METASD_STATUS_NONFINITE : 0u;
-                const float nma = -mg.Ma * c, nmb = -mg.Mb * c;
-                bool accepted = false;
-                if (pair2) {
-                    // lane j2 holds this position's token; every lane evaluates it on the broadcast values
-                    const int x = __shfl_sync(0xFFFFFFFFu, h_tok, j2);
-                    const float xa = __shfl_sync(0xFFFFFFFFu, h_xa, j2), xb = __shfl_sync(0xFFFFFFFFu, h_xb, j2);
-                    const float u = __shfl_sync(0xFFFFFFFFu, h_u, j2);
-                    float p_x = 0.f, q_x = 0.f;
-                    uint32_t fl = rowflag;
-                    if (!rowflag) {
-                        if (x < 0 || x >= V) {
-                            fl |= METASD_STATUS_TOKEN_OOR;
-                        } else {
-                            p_x = ex2(fmaf(xa, c, nma)) / mg.Sa;
-                            q_x = ex2(fmaf(xb, c, nmb)) / mg.Sb;
-                            if (p.greedy) {
-                                accepted = x == mg.idx;
-                            } else {
-                                if (q_x == 0.f) fl |= METASD_STATUS_Q_ZERO;
-                                accepted = u * q_x < p_x;   // u < min(1, p/q) without the division
-                            }
-                        }
-                    }
-                    seq_flags |= fl;
-                    if (lane == j2) { r_acc = accepted ? 1 : 0; r_px = p_x; r_qx = q_x; r_rowflag = rowflag; }
-                }
-                // first rejection (Algorithm 4, "exit for loop") or the bonus position: the next token comes from here
-                int mode = 0;
-                if (n_acc < 0) {
-                    if (pair2 && !accepted) { n_acc = j2; mode = 1; }
-                    if (!pair2) { n_acc = k; mode = 2; seq_flags |= rowflag; }
-                    if (mode) {
-                        if (rowflag) {
-                            mode = 0;
-                        } else if (p.greedy) {
-                            token = mg.idx;
-                            mode = 0;
-                        }
-                    }
-                }
-                const float ud = __shfl_sync(0xFFFFFFFFu, h_ud, j2);
-                if (lane == 0) {
-                    RowConst rc;
-                    rc.nma = nma;
-                    rc.nmb = nmb;
-                    // q_v / p_v = 2^(yb - ya) sum_a / sum_b: the ratio of the sums folds into the draft row's offset
-                    rc.nmb_rel = nmb + log2f(mg.Sa / mg.Sb);
-                    rc.inv_sa = 1.0f / mg.Sa;
-                    rc.inv_sb = 1.0f / mg.Sb;
-                    rc.u_draw = ud;
-                    rc.mode = mode;
-                    rc.valid = rowflag ? 0 : 1;
-                    sh.rc[s2] = rc;
-                    mbar_arrive(&sh.rcbar[s2]);   // release: the streaming warps may start pass 2 of this item
-                }
+                // expect one record of 32 bytes from every CTA of the cluster (this one included)
+                if (lane == 0 && !*(volatile int32_t *)&sh.dead)
+                    mbar_arrive_expect_tx(&sh.xbar[par], (uint32_t)csize * EXCHANGE_BYTES);
             }
-            // ---- the CTA's record of pass 1's item goes to every CTA of the cluster
-            if (do1) {
-                wait_bar(sh, &sh.wbar[s1], ph1, p.status);
-                const Merged mc = merge_records(sh.wrec[s1], ncw, lane, c);
-                if (lane < csize) {
-                    const uint32_t dst = map_to_rank(smem_addr(&sh.exch[u1][rank]), (uint32_t)lane);
-                    const uint32_t bar = map_to_rank(smem_addr(&sh.xbar[u1]), (uint32_t)lane);
-                    st_async_16(dst, bar, __float_as_uint(mc.Ma), __float_as_uint(mc.Sa), __float_as_uint(mc.Mb),
-                                __float_as_uint(mc.Sb));
-                    st_async_16(dst + 16, bar, (uint32_t)mc.idx, 0u, 0u, 0u);
-                }
-            }
-        } else {
-            if (do1) {
-                // ---- pass 1: statistics of this item's row slices out of shared memory
+
+            // ---- pass 1: statistics of this item's slices, chunk by chunk as the copies land
+            {
                 Exchange wr;
                 int v_t;
-                const int cb = c1 + 1 == g.n_slot ? 0 : c1 + 1;
-                const unsigned char *slot_a = ring + (size_t)c1 * g.slot_bytes, *slot_b = ring + (size_t)cb * g.slot_bytes;
-                wait_bar(sh, &sh.full[c1], c1par, p.status);
-                if (pair1) {
-                    wait_bar(sh, &sh.full[cb], cb == 0 ? c1par ^ 1u : c1par, p.status);
-                    stats_rows<LT, true>(slot_a, slot_b, my_vecs, ct, ncomp, trips, c, p.greedy != 0, wr.max_a, wr.sum_a, v_t,
-                                         wr.max_b, wr.sum_b);
-                } else {
-                    stats_rows<LT, false>(slot_a, slot_b, my_vecs, ct, ncomp, trips, c, p.greedy != 0, wr.max_a, wr.sum_a, v_t,
-                                          wr.max_b, wr.sum_b);
-                }
+                if (pair)
+                    stats_rows<LT, true>(sh, p.status, slot_a, slot_b, par_a, par_b, g.chunk_shift, my_vecs, tid, nthr, trips, c,
+                                         wr.max_a, wr.sum_a, v_t, wr.max_b, wr.sum_b);
+                else
+                    stats_rows<LT, false>(sh, p.status, slot_a, slot_b, par_a, par_b, g.chunk_shift, my_vecs, tid, nthr, trips, c,
+                                          wr.max_a, wr.sum_a, v_t, wr.max_b, wr.sum_b);
                 int cand = INT_MAX;
-                if (v_t >= 0) {   // first index of the maximum inside the vector in which this lane met it
+                if (p.greedy && v_t >= 0) {   // first index of the maximum inside the vector in which this lane met it
                     float x[VEC];
                     Logit<LT>::unpack(*reinterpret_cast<const uint4 *>(slot_a + (size_t)v_t * 16), x);
 #pragma unroll
@@ -793,90 +708,142 @@ __global__ void __launch_bounds__(FUSED_MAX_THREADS, 1) fused_round_kernel(const
                 wr.sum_b = warp_sum_f(wr.sum_b);
                 if (lane == 0) {
                     wr.pad[0] = wr.pad[1] = wr.pad[2] = 0;
-                    sh.wrec[s1][warp - 1] = wr;
-                    mbar_arrive(&sh.wbar[s1]);
+                    sh.wrec[warp] = wr;
                 }
             }
-            if (do2) {
-                // ---- pass 2: sum_v min(p_v, q_v) of this warp's logits
-                wait_bar(sh, &sh.rcbar[s2], ph2, p.status);
-                if (pair2) {
-                    const RowConst rc = sh.rc[s2];
-                    float acc = 0.f;
-                    if (rc.valid) acc = min_rows<LT>(a2, d2, my_vecs, ct, ncomp, c, rc.nma, rc.nmb_rel) * rc.inv_sa;
-                    acc = warp_sum_f(acc);
-                    if (lane == 0) sh.pmin[j2][warp - 1] = acc;
+            par_a ^= 1u;
+            if (pair) par_b ^= 1u;
+            __syncthreads();
+
+            // ---- the CTA's record goes to every CTA of the cluster (asynchronous stores that complete on
+            //      the receiver's barrier); then wait for all the records addressed to this CTA
+            if (warp == 0) {
+                const Merged mc = merge_records(sh.wrec, nw, lane, c);
+                if (lane < csize) {
+                    const uint32_t dst = map_to_rank(smem_addr(&sh.exch[par][rank]), (uint32_t)lane);
+                    const uint32_t bar = map_to_rank(smem_addr(&sh.xbar[par]), (uint32_t)lane);
+                    st_async_16(dst, bar, __float_as_uint(mc.Ma), __float_as_uint(mc.Sa), __float_as_uint(mc.Mb),
+                                __float_as_uint(mc.Sb));
+                    st_async_16(dst + 16, bar, (uint32_t)mc.idx, 0u, 0u, 0u);
                 }
             }
-        }
-        if (do2) {
-            const int mode = sh.rc[s2].mode;   // alike in every thread of the cluster; the control warp wrote it
+            wait_bar(sh, &sh.xbar[par], (item >> 1) & 1u, p.status);
+            const Merged mg = merge_records(sh.exch[par], csize, lane, c);
+            // NaN or +Inf anywhere makes the sum NaN; an all -Inf row leaves it 0
+            const bool bad_a = !(mg.Sa > 0.f) || !(mg.Sa < INFINITY) || !(mg.Ma < INFINITY);
+            const bool bad_b = pair && (!(mg.Sb > 0.f) || !(mg.Sb < INFINITY) || !(mg.Mb < INFINITY));
+            const uint32_t rowflag = (bad_a || bad_b) ? METASD_STATUS_NONFINITE : 0u;
+            RowConst rc;
+            rc.nma = -mg.Ma * c;
+            rc.nmb = -mg.Mb * c;
+            // q_v / p_v = 2^(yb - ya) sum_a / sum_b: the ratio of the sums folds into the draft row's offset
+            rc.nmb_rel = rc.nmb + log2f(mg.Sa / mg.Sb);
+            rc.inv_sa = 1.0f / mg.Sa;
+            rc.inv_sb = 1.0f / mg.Sb;
+            rc.u_draw = sh.h_ud[j];
+
+            // ---- pass 2: sum_v min(p_v, q_v) of this warp's logits; the accept test of Algorithm 4 (lines 7-8),
+            //      evaluated alike by every thread of the cluster
+            bool accepted = false;
+            if (pair) {
+                float acc = 0.f;
+                if (!rowflag) acc = min_rows<LT>(slot_a, slot_b, my_vecs, tid, nthr, c, rc.nma, rc.nmb_rel) * rc.inv_sa;
+                acc = warp_sum_f(acc);
+                if (lane == 0) sh.pmin[j][warp] = acc;
+
+                const int x = sh.h_tok[j];
+                float p_x = 0.f, q_x = 0.f;
+                uint32_t fl = rowflag;
+                if (!rowflag) {
+                    if (x < 0 || x >= V) {
+                        fl |= METASD_STATUS_TOKEN_OOR;
+                    } else {
+                        p_x = ex2(fmaf(sh.h_xa[j], c, rc.nma)) / mg.Sa;
+                        q_x = ex2(fmaf(sh.h_xb[j], c, rc.nmb)) / mg.Sb;
+                        if (p.greedy) {
+                            accepted = x == mg.idx;
+                        } else {
+                            if (q_x == 0.f) fl |= METASD_STATUS_Q_ZERO;
+                            accepted = sh.h_u[j] * q_x < p_x;   // u < min(1, p/q) without the division
+                        }
+                    }
+                }
+                seq_flags |= fl;
+                if (tid == 0) {
+                    sh.r_acc[j] = accepted ? 1 : 0;
+                    sh.r_px[j] = p_x;
+                    sh.r_qx[j] = q_x;
+                    sh.r_rowflag[j] = rowflag;
+                }
+            }
+
+            // ---- first rejection (Algorithm 4, "exit for loop") or the bonus position: emit the next token
+            int mode = 0;
+            if (n_acc < 0) {
+                if (pair && !accepted) { n_acc = j; mode = 1; }
+                if (!pair) { n_acc = k; mode = 2; seq_flags |= rowflag; }
+                if (mode) {
+                    if (rowflag) {
+                        mode = 0;
+                    } else if (p.greedy) {
+                        token = mg.idx;
+                        mode = 0;
+                    }
+                }
+            }
             if (mode) {
-                bool ok = cluster_draw<LT>(sh, sh.rc[s2], a2, d2, mode, c, my_vecs, vec0, rank, csize, ncw);
+                // the draw reads vectors this thread has not read before: see every chunk's copy complete first
+                for (int ch = 0; ch < n_chunk; ++ch) {
+                    wait_bar(sh, &sh.full[0][ch], par_a ^ 1u, p.status);
+                    if (pair) wait_bar(sh, &sh.full[1][ch], par_b ^ 1u, p.status);
+                }
+                bool ok = cluster_draw<LT>(sh, rc, slot_a, slot_b, mode, c, my_vecs, vec0, rank, csize, nw);
                 if (!ok && mode == 1)   // p == q in fp32 yet rejected: draw from p
-                    ok = cluster_draw<LT>(sh, sh.rc[s2], a2, d2, 2, c, my_vecs, vec0, rank, csize, ncw);
+                    ok = cluster_draw<LT>(sh, rc, slot_a, slot_b, 2, c, my_vecs, vec0, rank, csize, nw);
                 drew = ok;
             }
-            if (!pair2) {
-                // ---- end of the sequence: gather sum_v min(p, q) per position in rank 0
-                __syncthreads();
-                if (control && lane < k) {
-                    double s = 0.0;
-                    for (int w = 0; w < ncw; ++w) s += (double)sh.pmin[lane][w];
-                    st_cluster(map_to_rank(smem_addr(&sh.cta_min[lane][rank]), 0), s);
-                }
-                cluster_sync_all();
-                if (rank == 0 && control) {
-                    double smin = 0.0;
-                    if (lane < k) {
-                        for (int r = 0; r < csize; ++r) smin += sh.cta_min[lane][r];
-                        if (r_rowflag) smin = 0.0;
-                    }
-                    double sum_align = 0.0;
-                    for (int j = 0; j < k; ++j) sum_align += __shfl_sync(0xFFFFFFFFu, smin, j);
-                    // Definition 2: 1 - mean_j d_TV; block efficiency: N_acc / N_max
-                    const double r = p.reward_kind == METASD_REWARD_BE ? (double)n_acc / (double)k : sum_align / (double)k;
-                    if (p.diag && lane < k) {
-                        metasd_diag dg;
-                        dg.p_x = r_px;
-                        dg.q_x = r_qx;
-                        dg.D = r_rowflag ? 1.f : (float)(1.0 - smin);
-                        dg.u = h_u;
-                        dg.accept = r_acc;
-                        p.diag[(size_t)b2 * k + lane] = dg;
-                    }
-                    if (lane == 0) {
-                        p.accepted_len[b2] = n_acc;
-                        p.next_token[b2] = drew ? sh.token : token;
-                        p.reward[b2] = (float)r;
-                        if (seq_flags) atomicOr(p.status, seq_flags);
-                    }
-                    warp_bandit(p, b2, h_t, h_arm, r);
-                }
+            __syncthreads();   // every warp is done with the slices: the next item's copies may overwrite them
+            if (tid == 0) {
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                issue_item();
             }
-            // ---- pass 2's slots go back to the ring: the streaming warps sign off, the control warp refills
-            if (!control) {
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&sh.ebar[s2]);
-            } else {
-                wait_bar(sh, &sh.ebar[s2], ph2, p.status);
-                if (lane == 0) {
-                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                    issue_one();
-                    if (pair2) issue_one();
-                }
-                __syncwarp();
-            }
-            c2 += pair2 ? 2 : 1;
-            if (c2 >= g.n_slot) c2 -= g.n_slot;
-            if (++u2 == 3) { u2 = 0; x2par ^= 1u; }
-            if (++j2 > k) { j2 = 0; b2 += ncl; }
         }
-        if (do1) {
-            c1 += pair1 ? 2 : 1;
-            if (c1 >= g.n_slot) { c1 -= g.n_slot; c1par ^= 1u; }
-            if (++u1 == 3) u1 = 0;
-            if (++j1 > k) j1 = 0;
+
+        // ---- end of the sequence: gather sum_v min(p, q) per position in rank 0
+        if (warp == 0 && lane < k) {
+            double s = 0.0;
+            for (int w = 0; w < nw; ++w) s += (double)sh.pmin[lane][w];
+            st_cluster(map_to_rank(smem_addr(&sh.cta_min[lane][rank]), 0), s);
+        }
+        cluster_sync_all();
+        if (rank == 0 && warp == 0) {
+            double smin = 0.0;
+            uint32_t rf = 0;
+            if (lane < k) {
+                for (int r = 0; r < csize; ++r) smin += sh.cta_min[lane][r];
+                rf = sh.r_rowflag[lane];
+                if (rf) smin = 0.0;
+            }
+            double sum_align = 0.0;
+            for (int j = 0; j < k; ++j) sum_align += __shfl_sync(0xFFFFFFFFu, smin, j);
+            // Definition 2: 1 - mean_j d_TV; block efficiency: N_acc / N_max
+            const double r = p.reward_kind == METASD_REWARD_BE ? (double)n_acc / (double)k : sum_align / (double)k;
+            if (p.diag && lane < k) {
+                metasd_diag dg;
+                dg.p_x = sh.r_px[lane];
+                dg.q_x = sh.r_qx[lane];
+                dg.D = rf ? 1.f : (float)(1.0 - smin);
+                dg.u = sh.h_u[lane];
+                dg.accept = sh.r_acc[lane];
+                p.diag[(size_t)b * k + lane] = dg;
+            }
+            if (lane == 0) {
+                p.accepted_len[b] = n_acc;
+                p.next_token[b] = drew ? sh.token : token;
+                p.reward[b] = (float)r;
+                if (seq_flags) atomicOr(p.status, seq_flags);
+            }
+            warp_bandit(p, b, sh.h_t, sh.h_arm, r);
         }
     }
 
@@ -898,8 +865,8 @@ const void *kernel_for(int dtype)
                                 : reinterpret_cast<const void *>(&fused_round_kernel<float>);
 }
 
-// Geometry for cluster size C, or false when the row does not fit.
-bool geometry(int dtype, int V, int C, int smem_optin, FusedPlan *pl)
+// Geometry for cluster size C, or false when a slice pair does not fit half an SM's shared memory.
+bool geometry(int dtype, int V, int C, int smem_per_sm, FusedPlan *pl)
 {
     const size_t row_bytes = (size_t)V * (dtype == METASD_BF16 ? 2 : 4);
     if (row_bytes % 16 != 0) return false;
@@ -908,24 +875,25 @@ bool geometry(int dtype, int V, int C, int smem_optin, FusedPlan *pl)
     const int n_vec_cta = (n_vec_row + C - 1) / C;
     if ((size_t)(C - 1) * n_vec_cta >= (size_t)n_vec_row) return false;   // an empty last rank: a smaller C serves better
     const int slot_bytes = n_vec_cta * 16;
-    int n_slot = (smem_optin - FUSED_SMEM_RESERVE) / slot_bytes;
-    if (n_slot > FUSED_MAX_SLOTS) n_slot = FUSED_MAX_SLOTS;
-    if (n_slot < FUSED_MIN_SLOTS) return false;
-    // streaming warps: the count that divides the slice with the least padding (the larger count on ties),
-    // plus the control warp
+    // two CTAs per SM; each CTA also pays 1 KB that the system reserves
+    const int budget = smem_per_sm / 2 - 1024 - FUSED_STATIC_SMEM;
+    if (2 * slot_bytes > budget) return false;
+    // warps: the count that covers the slice with the least padding (the larger count on ties)
     int best_w = 0;
     long best_cost = 0;
-    for (int w = FUSED_MAX_WARPS - 1; w >= 1; --w) {
+    for (int w = FUSED_MAX_THREADS / 32; w >= 2; --w) {
         const long cost = (long)(w * 32) * ((n_vec_cta + w * 32 - 1) / (w * 32));
         if (!best_w || cost < best_cost) { best_w = w; best_cost = cost; }
     }
+    int shift = 0;
+    while ((FUSED_CHUNKS << shift) < n_vec_cta) ++shift;
     pl->cluster = C;
-    pl->threads = (best_w + 1) * 32;
+    pl->threads = best_w * 32;
     pl->n_vec_row = n_vec_row;
     pl->n_vec_cta = n_vec_cta;
-    pl->n_slot = n_slot;
+    pl->n_slot = shift;   // log2 of the vectors per chunk
     pl->slot_bytes = slot_bytes;
-    pl->smem_bytes = (size_t)n_slot * slot_bytes;
+    pl->smem_bytes = (size_t)2 * slot_bytes;
     pl->work_per_item = n_vec_cta;
     pl->max_clusters = 0;
     return true;
@@ -944,21 +912,21 @@ bool fused_supported(int dtype, int V, int k)
     if (k < 1 || k > 16) return false;
     FusedPlan pl;
     for (int C = 1; C <= FUSED_MAX_CLUSTER; ++C)
-        if (geometry(dtype, V, C, 227 * 1024, &pl)) return true;
+        if (geometry(dtype, V, C, 228 * 1024, &pl)) return true;
     return false;
 }
 
-// Chooses the cluster size for this device: for every size that fits, ask the occupancy calculator how
-// many clusters are co-resident (GPC shapes decide) and take the least estimated time for a full batch.
+// Chooses the cluster size for this device: the smallest for which two CTAs fit an SM, and asks the occupancy
+// calculator how many clusters are co-resident (GPC shapes decide).
 // METASD_FUSED_CLUSTER / METASD_FUSED_THREADS (environment) pin the choice for tuning runs.
 cudaError_t fused_prepare(int device, int dtype, int V, int max_batch, FusedPlan *plan)
 {
     plan->cluster = 0;
-    int smem_optin = 0;
-    cudaError_t e = cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device);
+    int smem_per_sm = 0;
+    cudaError_t e = cudaDeviceGetAttribute(&smem_per_sm, cudaDevAttrMaxSharedMemoryPerMultiprocessor, device);
     if (e != cudaSuccess) return e;
     const void *fn = kernel_for(dtype);
-    e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin - FUSED_SMEM_RESERVE);
+    e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_per_sm / 2 - 1024 - FUSED_STATIC_SMEM);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
     if (e != cudaSuccess) return e;
@@ -967,7 +935,7 @@ cudaError_t fused_prepare(int device, int dtype, int V, int max_batch, FusedPlan
     for (int C = 1; C <= FUSED_MAX_CLUSTER; ++C) {
         if (pin_c && C != pin_c) continue;
         FusedPlan pl;
-        if (!geometry(dtype, V, C, smem_optin, &pl)) continue;
+        if (!geometry(dtype, V, C, smem_per_sm, &pl)) continue;
         if (pin_t >= 64 && pin_t <= FUSED_MAX_THREADS && pin_t % 32 == 0) pl.threads = pin_t;
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(C);
@@ -989,10 +957,11 @@ cudaError_t fused_prepare(int device, int dtype, int V, int max_batch, FusedPlan
         // per item: the two passes over the slice plus a fixed cost for barriers and exchanges
         const double cost = waves * ((double)pl.work_per_item + 300.0);
         if (!plan->cluster || cost < best) { *plan = pl; best = cost; }
+        if (!pin_c) break;   // the smallest size that fits: the largest slices, the fewest exchange partners
     }
     if (plan->cluster && env_int("METASD_FUSED_VERBOSE", 0))
-        fprintf(stderr, "metasd fused plan: V=%d cluster=%d threads=%d vectors/cta=%d slots=%d x %d B, %d clusters co-resident\n",
-                V, plan->cluster, plan->threads, plan->n_vec_cta, plan->n_slot, plan->slot_bytes, plan->max_clusters);
+        fprintf(stderr, "metasd fused plan: V=%d cluster=%d threads=%d vectors/cta=%d (chunks of %d), %zu B shared, %d clusters co-resident\n",
+                V, plan->cluster, plan->threads, plan->n_vec_cta, 1 << plan->n_slot, plan->smem_bytes, plan->max_clusters);
     return plan->cluster ? cudaSuccess : cudaErrorNotSupported;
 }
 
@@ -1001,8 +970,8 @@ cudaError_t launch_fused(const VerifyParams &p, int dtype, const FusedPlan &plan
     FusedGeom g;
     g.n_vec_row = plan.n_vec_row;
     g.n_vec_cta = plan.n_vec_cta;
-    g.n_slot = plan.n_slot;
     g.slot_bytes = plan.slot_bytes;
+    g.chunk_shift = plan.n_slot;
     const int n_clusters = p.batch < plan.max_clusters ? p.batch : plan.max_clusters;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(n_clusters * plan.cluster));

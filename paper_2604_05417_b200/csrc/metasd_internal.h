@@ -64,7 +64,7 @@ struct FusedPlan {
     int32_t threads;       // threads per CTA
     int32_t n_vec_row;     // 16-byte vectors per logit row
     int32_t n_vec_cta;     // vectors of a row owned by one CTA
-    int32_t n_slot;        // ring slots of slot_bytes each
+    int32_t n_slot;        // log2 of the vectors per chunk of a slice
     int32_t slot_bytes;
     int32_t max_clusters;  // co-resident clusters on the device
     size_t smem_bytes;     // dynamic shared memory of the launch
