@@ -22,6 +22,11 @@ struct metasd_ctx {
     float *stage_reward;
     bool fused_ready;
     FusedPlan plan;
+    // split streaming path
+    int grp_size, grp_ctas;
+    GroupRecord *grp_rec;
+    double *grp_min;
+    uint32_t *grp_count;
 };
 
 namespace {
@@ -68,6 +73,7 @@ void free_all(metasd_ctx *c)
     cudaFree(c->st.win_arm); cudaFree(c->st.win_reward); cudaFree(c->stats); cudaFree(c->status);
     cudaFree(c->stage_target); cudaFree(c->stage_draft); cudaFree(c->stage_tokens);
     cudaFree(c->stage_acc); cudaFree(c->stage_tok); cudaFree(c->stage_reward);
+    cudaFree(c->grp_rec); cudaFree(c->grp_min); cudaFree(c->grp_count);
 }
 
 }  // namespace
@@ -132,6 +138,14 @@ int metasd_init(metasd_ctx **out, const metasd_config *cfg)
         alloc((void **)&c->stage_acc, B * sizeof(int32_t));
         alloc((void **)&c->stage_tok, B * sizeof(int32_t));
         alloc((void **)&c->stage_reward, B * sizeof(float));
+    }
+    if (e == cudaSuccess) {
+        e = split_prepare(cfg->device, cfg->logit_dtype, cfg->vocab, &c->grp_ctas, &c->grp_size);
+        if (e == cudaSuccess && c->grp_size > 1) {
+            alloc((void **)&c->grp_rec, B * kp1 * c->grp_size * sizeof(GroupRecord));
+            alloc((void **)&c->grp_min, B * kp1 * c->grp_size * sizeof(double));
+            alloc((void **)&c->grp_count, B * kp1 * sizeof(uint32_t));
+        }
     }
     if (e == cudaSuccess) e = cudaMemset(c->status, 0, sizeof(uint32_t));
     if (e == cudaSuccess) e = launch_reset(c->st, cfg->max_batch, cfg->n_drafters, cfg->window, nullptr, cfg->max_batch, 0);
@@ -209,6 +223,8 @@ int metasd_verify(metasd_ctx *ctx, int32_t batch, int32_t k, const void *target_
     p.seed = seed; p.beta = cfg.beta; p.gamma = cfg.gamma;
     p.accepted_len = accepted_len; p.next_token = next_token; p.reward = reward; p.diag = diag;
     p.st = ctx->st; p.stats = ctx->stats; p.status = ctx->status;
+    p.grp_size = ctx->grp_size; p.grp_ctas = ctx->grp_ctas;
+    p.grp_rec = ctx->grp_rec; p.grp_min = ctx->grp_min; p.grp_count = ctx->grp_count;
     const size_t row_bytes = (size_t)cfg.vocab * logit_size(cfg.logit_dtype);
     // with a pointer table the per-drafter bases are not visible here: the caller's contract is that
     // they are aligned like the target

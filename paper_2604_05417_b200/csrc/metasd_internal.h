@@ -18,6 +18,13 @@ struct RowStats {
     uint32_t flags;       // METASD_STATUS_* of this row pair
 };
 
+// What one CTA of a group publishes about its part of a row pair (split streaming path).
+struct GroupRecord {
+    float max_a, sum_a, max_b, sum_b;
+    int32_t argmax_a;
+    int32_t pad[3];
+};
+
 // Bandit state of all sequences, structure of arrays in device memory.
 struct BanditState {
     int32_t *t;          // [B] rounds completed
@@ -54,6 +61,12 @@ struct VerifyParams {
     RowStats *stats;   // [batch, k+1]
     uint32_t *status;
     int32_t vector_ok; // rows are 16-byte aligned and a whole number of 16-byte vectors
+    // split streaming path: grp_size CTAs share a row pair (0: one CTA per row pair)
+    int32_t grp_size;
+    int32_t grp_ctas;        // CTAs of the launch (co-resident)
+    GroupRecord *grp_rec;    // [batch * (k + 1), grp_size]
+    double *grp_min;         // [batch * (k + 1), grp_size] partial sums of min(p, q)
+    uint32_t *grp_count;     // [batch * (k + 1)] arrivals, cleared before every launch
 };
 
 // streaming path (metasd_streaming.cu)
@@ -74,6 +87,9 @@ bool fused_supported(int dtype, int V, int k);
 cudaError_t fused_prepare(int device, int dtype, int V, int max_batch, FusedPlan *plan);
 cudaError_t launch_fused(const VerifyParams &p, int dtype, const FusedPlan &plan, cudaStream_t stream,
                          uint64_t *launches);
+// how many CTAs of the split kernel are co-resident, and how many of them should share a row pair so that
+// the rows in flight stay inside L2 (1: not worth splitting)
+cudaError_t split_prepare(int device, int dtype, int V, int *resident_ctas, int *group_size);
 // small state kernels (metasd_streaming.cu)
 cudaError_t launch_select(const BanditState &st, int batch, int32_t *arm_out, cudaStream_t stream);
 cudaError_t launch_reset(const BanditState &st, int max_batch, int K, int tau, const int32_t *seq_ids,

@@ -1,5 +1,9 @@
 // Streaming path of the MetaSD verify round: works for every shape.
 //
+//   K1s split_row_stats_kernel  the same statistics as K1 with grp_size co-resident CTAs per row pair, each on its
+//                          own part of the vocabulary: they exchange (max, sum, arg-max) records through global
+//                          memory between the two sweeps.  Few enough row pairs are then in flight for the second
+//                          sweep to be served by L2 instead of HBM.  Used for 16-byte aligned rows when splitting pays.
 //   K1  row_stats_kernel   one CTA per (sequence b, position j): softmax statistics of the target
 //                          row and the draft row with an online maximum, the target arg-max, then
 //                          sum_v min(p_v, q_v) = 1 - d_TV(p_j, q_j) (Definition 2) in a second
@@ -8,6 +12,8 @@
 //                          lines 7-8), first rejection, inverse-CDF draw of the correction token from
 //                          max(0, p - q) or of the bonus token from p (lines 11-12), the reward, the
 //                          bandit update and the next round's arm (Algorithm 2, lines 7-10).
+#include <stdlib.h>
+
 #include "metasd_device.cuh"
 
 namespace metasd {
@@ -147,6 +153,237 @@ __global__ void __launch_bounds__(K1_THREADS) row_stats_kernel(const VerifyParam
         r.flags = flags;
         p.stats[(size_t)b * (p.k + 1) + j] = r;
     }
+}
+
+// -------------------------------------------------------------------------------------------
+// K1s
+// -------------------------------------------------------------------------------------------
+constexpr int KS_THREADS = 512;
+constexpr uint32_t KS_SPIN_LIMIT = 1u << 22;   // polls of 64 ns: a quarter of a second
+
+// Adds 1 without waiting for the result; the thread's earlier writes are visible to whoever sees the new count.
+__device__ __forceinline__ void red_release_inc(uint32_t *p)
+{
+    asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p) : "memory");
+}
+__device__ __forceinline__ uint32_t ld_acquire(const uint32_t *p)
+{
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// Warp 0 of every CTA only communicates: while the other warps sweep, it publishes the CTA's record of one row
+// pair (fence + counter), waits (bounded) for the group's records of the row pair whose second sweep comes next,
+// merges them, and adds up and publishes the partial sums of min(p, q).  The global-memory round trips of the
+// exchange therefore overlap the sweeps.  The first sweep of the NEXT row pair runs before the second sweep of
+// the current one, so a group's records have a whole sweep's time to arrive.
+template <typename LT>
+__global__ void __launch_bounds__(KS_THREADS, 3) split_row_stats_kernel(const VerifyParams p)
+{
+    constexpr int VEC = Logit<LT>::VEC;
+    constexpr int NWARP = KS_THREADS / 32;          // warp 0 + NWARP - 1 sweeping warps
+    constexpr int NSWEEP = KS_THREADS - 32;         // sweeping threads
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int st = tid - 32;                        // index among the sweeping threads
+    const int V = p.V, G = p.grp_size;
+    const float c = p.c;
+    const int n_groups = gridDim.x / G, grp = blockIdx.x / G, g = blockIdx.x - grp * G;
+    const int nvec = V / VEC, per = (nvec + G - 1) / G;
+    const int v_lo = min(g * per, nvec), v_hi = min(v_lo + per, nvec);   // this CTA's part of every row
+    __shared__ MaxSum sh_a[NWARP], sh_b[NWARP];
+    __shared__ ArgMax sh_am[NWARP];
+    __shared__ double sh_min[NWARP];
+    __shared__ float sh_bcast[5];      // merged statistics of the row pair in its second sweep
+    __shared__ int sh_arg;
+    const int n_items = p.batch * (p.k + 1);
+
+    auto row_ptrs = [&](int item, const LT *&a, const LT *&d, bool &pair) {
+        const int b = item / (p.k + 1), j = item - b * (p.k + 1);
+        pair = j < p.k;
+        a = reinterpret_cast<const LT *>(p.target) + ((size_t)b * (p.k + 1) + j) * V;
+        d = pair ? draft_rows<LT>(p, b) + ((size_t)b * p.k + j) * V : nullptr;
+    };
+    // ---- sweeping warps: online (max, sum) of both rows, arg-max of the target row, over this CTA's part
+    auto first_sweep = [&](int item) {
+        const LT *a, *d;
+        bool pair;
+        row_ptrs(item, a, d, pair);
+        MaxSum sa = {METASD_NEG_BIG, 0.f}, sb = {METASD_NEG_BIG, 0.f};
+        ArgMax am = {METASD_NEG_BIG, 0x7FFFFFFF};
+        for (int i = v_lo + st; i < v_hi; i += NSWEEP) {
+            float xa[VEC], xb[VEC];
+            Logit<LT>::unpack(ld_stream(reinterpret_cast<const uint4 *>(a) + i), xa);
+            if (pair) Logit<LT>::unpack(ld_stream(reinterpret_cast<const uint4 *>(d) + i), xb);
+            float cm = xa[0];
+#pragma unroll
+            for (int e = 1; e < VEC; ++e) cm = fmaxf(cm, xa[e]);
+            if (cm > sa.m) {
+                sa.s *= ex2((sa.m - cm) * c);
+                sa.m = cm;
+                int first = 0;
+#pragma unroll
+                for (int e = VEC - 1; e >= 0; --e)
+                    if (xa[e] == cm) first = e;
+                am.v = cm;
+                am.i = i * VEC + first;
+            }
+            const float nma = -sa.m * c;
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) sa.s += ex2(fmaf(xa[e], c, nma));
+            if (pair) {
+                float bm = xb[0];
+#pragma unroll
+                for (int e = 1; e < VEC; ++e) bm = fmaxf(bm, xb[e]);
+                if (bm > sb.m) {
+                    sb.s *= ex2((sb.m - bm) * c);
+                    sb.m = bm;
+                }
+                const float nmb = -sb.m * c;
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) sb.s += ex2(fmaf(xb[e], c, nmb));
+            }
+        }
+        sa = warp_merge(sa, c);
+        sb = warp_merge(sb, c);
+        am = warp_argmax(am);
+        if (lane == 0) { sh_a[warp] = sa; sh_b[warp] = sb; sh_am[warp] = am; }
+    };
+    // ---- sweeping warps: sum_v min(p_v, q_v) = (1 / sum_a) sum_v 2^min(ya_v, yb_v) over this CTA's part
+    auto second_sweep = [&](int item) {
+        const LT *a, *d;
+        bool pair;
+        row_ptrs(item, a, d, pair);
+        double w = 0.0;
+        if (pair) {
+            const float nma = -sh_bcast[0] * c, nmb = sh_bcast[4], sum_a = sh_bcast[1];
+            float acc = 0.f;
+            for (int i = v_lo + st; i < v_hi; i += NSWEEP) {
+                float xa[VEC], xb[VEC];
+                Logit<LT>::unpack(ld_stream(reinterpret_cast<const uint4 *>(a) + i), xa);
+                Logit<LT>::unpack(ld_stream(reinterpret_cast<const uint4 *>(d) + i), xb);
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) acc += ex2(fminf(fmaf(xa[e], c, nma), fmaf(xb[e], c, nmb)));
+            }
+            w = warp_sum((double)(acc / sum_a));
+        }
+        if (lane == 0) sh_min[warp] = w;
+    };
+    // ---- warp 0: the CTA's record of a first sweep goes to global memory
+    auto publish_record = [&](int item) {
+        MaxSum ra = (lane >= 1 && lane < NWARP) ? sh_a[lane] : MaxSum{METASD_NEG_BIG, 0.f};
+        MaxSum rb = (lane >= 1 && lane < NWARP) ? sh_b[lane] : MaxSum{METASD_NEG_BIG, 0.f};
+        ArgMax rm = (lane >= 1 && lane < NWARP) ? sh_am[lane] : ArgMax{METASD_NEG_BIG, 0x7FFFFFFF};
+        ra = warp_merge(ra, c);
+        rb = warp_merge(rb, c);
+        rm = warp_argmax(rm);
+        if (lane == 0) {
+            GroupRecord r;
+            r.max_a = ra.m; r.sum_a = ra.s; r.max_b = rb.m; r.sum_b = rb.s; r.argmax_a = rm.i;
+            r.pad[0] = r.pad[1] = r.pad[2] = 0;
+            p.grp_rec[(size_t)item * G + g] = r;
+            red_release_inc(&p.grp_count[item]);
+        }
+    };
+    // ---- warp 0: wait (bounded) for the group's records of a row pair and merge them for its second sweep
+    auto merge_group = [&](int item) {
+        if (lane == 0) {
+            uint32_t it = 0;
+            while (ld_acquire(&p.grp_count[item]) < (uint32_t)G) {
+                if (++it > KS_SPIN_LIMIT) { atomicOr(p.status, METASD_STATUS_TIMEOUT); break; }
+                __nanosleep(64);
+            }
+        }
+        __syncwarp();
+        MaxSum ga = {METASD_NEG_BIG, 0.f}, gb = {METASD_NEG_BIG, 0.f};
+        ArgMax gm = {METASD_NEG_BIG, 0x7FFFFFFF};
+        if (lane < G) {
+            const int4 *src = reinterpret_cast<const int4 *>(p.grp_rec + (size_t)item * G + lane);
+            const int4 lo = __ldcg(src), hi = __ldcg(src + 1);
+            ga.m = __int_as_float(lo.x); ga.s = __int_as_float(lo.y);
+            gb.m = __int_as_float(lo.z); gb.s = __int_as_float(lo.w);
+            gm.v = ga.m; gm.i = hi.x;
+        }
+        ga = warp_merge(ga, c);
+        gb = warp_merge(gb, c);
+        gm = warp_argmax(gm);
+        if (lane == 0) {
+            sh_bcast[0] = ga.m; sh_bcast[1] = ga.s; sh_bcast[2] = gb.m; sh_bcast[3] = gb.s;
+            // q_v / p_v = 2^(yb - ya) sum_a / sum_b: the ratio of the sums folds into the draft row's offset
+            sh_bcast[4] = -gb.m * c + log2f(ga.s / gb.s);
+            sh_arg = gm.i;
+        }
+    };
+    // ---- warp 0: this CTA's part of sum min(p, q)
+    auto publish_min = [&](int item) {
+        if (lane == 0) {
+            double part = 0.0;
+            for (int i = 1; i < NWARP; ++i) part += sh_min[i];
+            p.grp_min[(size_t)item * G + g] = part;
+            red_release_inc(&p.grp_count[item]);
+        }
+    };
+    // ---- warp 0 of one CTA of the group (they take turns): once every part is in, add the parts up and write the
+    //      row pair's statistics
+    auto finalise = [&](int item, float max_a, float sum_a, float max_b, float sum_b, int arg) {
+        if (lane == 0) {
+            uint32_t it = 0;
+            while (ld_acquire(&p.grp_count[item]) < 2u * (uint32_t)G) {
+                if (++it > KS_SPIN_LIMIT) { atomicOr(p.status, METASD_STATUS_TIMEOUT); break; }
+                __nanosleep(64);
+            }
+            const bool pair = item % (p.k + 1) < p.k;
+            double total = 0.0;
+            for (int i = 0; i < G; ++i) total += __ldcg(p.grp_min + (size_t)item * G + i);
+            RowStats r;
+            r.max_a = max_a; r.sum_a = sum_a; r.max_b = max_b; r.sum_b = sum_b;
+            r.argmax_a = arg;
+            uint32_t flags = 0;
+            // NaN or +Inf anywhere makes the sum NaN; an all -Inf row leaves it 0
+            const bool bad_a = !(sum_a > 0.f) || !(sum_a < INFINITY) || !(max_a < INFINITY);
+            const bool bad_b = pair && (!(sum_b > 0.f) || !(sum_b < INFINITY) || !(max_b < INFINITY));
+            if (bad_a || bad_b) flags |= METASD_STATUS_NONFINITE;
+            r.sum_min = flags ? 0.0 : total;
+            r.flags = flags;
+            p.stats[item] = r;
+        }
+    };
+
+    // Group grp takes row pairs grp, grp + n_groups, ... in (sequence, position) order.
+    if (grp < n_items) {
+        if (warp != 0) first_sweep(grp);
+        __syncthreads();
+        if (warp == 0) publish_record(grp);
+    }
+    // warp 0: statistics of the row pair in its second sweep, and of the one before (for the finalising turn)
+    float m_a = 0.f, s_a = 0.f, m_b = 0.f, s_b = 0.f, pm_a = 0.f, ps_a = 0.f, pm_b = 0.f, ps_b = 0.f;
+    int arg = 0, parg = 0, prev = -1, turn = 0;
+    for (int item = grp; item < n_items; item += n_groups, ++turn) {
+        const int next = item + n_groups;
+        // phase A: first sweep of the next row pair | warp 0 prepares the second sweep of this one
+        if (warp != 0) {
+            if (next < n_items) first_sweep(next);
+        } else {
+            merge_group(item);
+            m_a = sh_bcast[0]; s_a = sh_bcast[1]; m_b = sh_bcast[2]; s_b = sh_bcast[3]; arg = sh_arg;
+        }
+        __syncthreads();
+        // phase B: second sweep of this row pair | warp 0 publishes the next one's record and, on its turn,
+        // writes the statistics of the previous row pair
+        if (warp != 0) {
+            second_sweep(item);
+        } else {
+            if (next < n_items) publish_record(next);
+            if (prev >= 0 && (turn - 1) % G == g) finalise(prev, pm_a, ps_a, pm_b, ps_b, parg);
+        }
+        __syncthreads();
+        // warp 0 publishes this row pair's partial sum while the others start the next phase A
+        if (warp == 0) {
+            publish_min(item);
+            prev = item; pm_a = m_a; ps_a = s_a; pm_b = m_b; ps_b = s_b; parg = arg;
+        }
+    }
+    if (warp == 0 && prev >= 0 && (turn - 1) % G == g) finalise(prev, pm_a, ps_a, pm_b, ps_b, parg);
 }
 
 // -------------------------------------------------------------------------------------------
@@ -396,7 +633,20 @@ template <typename LT>
 static cudaError_t launch_streaming_t(const VerifyParams &p, cudaStream_t stream, uint64_t *launches)
 {
     dim3 g1(p.k + 1, p.batch), g2(p.batch);
-    if (p.vector_ok) {
+    if (p.vector_ok && p.grp_size > 1) {
+        const int n_items = p.batch * (p.k + 1);
+        int n_groups = p.grp_ctas / p.grp_size;
+        if (n_groups > n_items) n_groups = n_items;
+        cudaError_t e = cudaMemsetAsync(p.grp_count, 0, (size_t)n_items * sizeof(uint32_t), stream);
+        if (e != cudaSuccess) return e;
+        // the CTAs of a group wait on one another: a cooperative launch guarantees that they are co-resident
+        VerifyParams q = p;
+        void *args[] = {&q};
+        e = cudaLaunchCooperativeKernel(reinterpret_cast<const void *>(&split_row_stats_kernel<LT>), dim3(n_groups * p.grp_size),
+                                        dim3(KS_THREADS), args, 0, stream);
+        if (e != cudaSuccess) return e;
+        epilogue_kernel<LT, true><<<g2, K2_THREADS, 0, stream>>>(p);
+    } else if (p.vector_ok) {
         row_stats_kernel<LT, true><<<g1, K1_THREADS, 0, stream>>>(p);
         epilogue_kernel<LT, true><<<g2, K2_THREADS, 0, stream>>>(p);
     } else {
@@ -411,6 +661,36 @@ cudaError_t launch_streaming(const VerifyParams &p, int dtype, cudaStream_t stre
 {
     if (dtype == METASD_BF16) return launch_streaming_t<__nv_bfloat16>(p, stream, launches);
     return launch_streaming_t<float>(p, stream, launches);
+}
+
+cudaError_t split_prepare(int device, int dtype, int V, int *resident_ctas, int *group_size)
+{
+    *resident_ctas = 0;
+    *group_size = 1;
+    int per_sm = 0, n_sm = 0, l2 = 0, coop = 0;
+    cudaError_t e;
+    if (dtype == METASD_BF16)
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, split_row_stats_kernel<__nv_bfloat16>, KS_THREADS, 0);
+    else
+        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, split_row_stats_kernel<float>, KS_THREADS, 0);
+    if (e != cudaSuccess) return e;
+    if ((e = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, device)) != cudaSuccess) return e;
+    if ((e = cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, device)) != cudaSuccess) return e;
+    if ((e = cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, device)) != cudaSuccess) return e;
+    if (!coop || per_sm < 1) return cudaSuccess;
+    const int resident = per_sm * n_sm;
+    // row-pair bytes in flight = resident CTAs x (row pair / group size); keep them within a third of L2
+    const double pair_bytes = 2.0 * V * (dtype == METASD_BF16 ? 2 : 4);
+    const char *pin = getenv("METASD_SPLIT_GROUP");
+    // measured on B200: the exchange costs more than the saved HBM traffic gains, so splitting is opt-in
+    // (METASD_SPLIT_GROUP); the L2-sized default would be ceil(resident * pair_bytes / (l2 / 3))
+    (void)pair_bytes; (void)l2;
+    int G = pin && *pin ? atoi(pin) : 1;
+    if (G < 1) G = 1;
+    if (G > 16) G = 16;
+    *resident_ctas = resident - resident % G;
+    *group_size = G;
+    return cudaSuccess;
 }
 
 // -------------------------------------------------------------------------------------------
