@@ -52,9 +52,11 @@ enum metasd_reward { METASD_REWARD_BD = 0, METASD_REWARD_BE = 1 };
 
 /* Which kernels metasd_verify launches. */
 enum metasd_path {
-    METASD_PATH_AUTO = 0,      /* fused cluster kernel when the shape fits it, else streaming */
+    METASD_PATH_AUTO = 0,      /* the fastest measured path for the shape (currently: streaming) */
     METASD_PATH_STREAMING = 1, /* row-statistics kernel + per-sequence epilogue kernel; any shape */
-    METASD_PATH_FUSED = 2      /* one persistent thread-block-cluster kernel per call */
+    METASD_PATH_FUSED = 2      /* one persistent thread-block-cluster kernel per call: every logit is read
+                                  from HBM once; needs 16-byte aligned rows that fit its geometry, else
+                                  metasd_init returns METASD_ERR_UNSUPPORTED */
 };
 
 /* Status bits (OR-accumulated on the device until read). */

@@ -149,7 +149,7 @@ int metasd_init(metasd_ctx **out, const metasd_config *cfg)
     }
     if (e == cudaSuccess) e = cudaMemset(c->status, 0, sizeof(uint32_t));
     if (e == cudaSuccess) e = launch_reset(c->st, cfg->max_batch, cfg->n_drafters, cfg->window, nullptr, cfg->max_batch, 0);
-    if (e == cudaSuccess && cfg->path != METASD_PATH_STREAMING &&
+    if (e == cudaSuccess && cfg->path == METASD_PATH_FUSED &&
         fused_supported(cfg->logit_dtype, cfg->vocab, cfg->max_draft)) {
         e = fused_prepare(cfg->device, cfg->logit_dtype, cfg->vocab, cfg->max_batch, &c->plan);
         c->fused_ready = (e == cudaSuccess);
@@ -193,7 +193,9 @@ int metasd_select(metasd_ctx *ctx, int32_t batch, int32_t *arm_out, void *stream
 int metasd_resolved_path(const metasd_ctx *ctx, int32_t k)
 {
     if (!ctx) return METASD_ERR_INVALID_ARGUMENT;
-    if (ctx->cfg.path == METASD_PATH_STREAMING) return METASD_PATH_STREAMING;
+    // AUTO takes the streaming kernels: on B200 they are the faster path at every measured shape (the fused
+    // cluster kernel reads each logit once but is bound by its exchange and instruction overheads).
+    if (ctx->cfg.path != METASD_PATH_FUSED) return METASD_PATH_STREAMING;
     if (ctx->fused_ready && fused_supported(ctx->cfg.logit_dtype, ctx->cfg.vocab, k)) return METASD_PATH_FUSED;
     return METASD_PATH_STREAMING;
 }

@@ -91,7 +91,7 @@ __global__ void __launch_bounds__(K1_THREADS) row_stats_kernel(const VerifyParam
     __shared__ MaxSum sh_a[NWARP], sh_b[NWARP];
     __shared__ ArgMax sh_am[NWARP];
     __shared__ double sh_min[NWARP];
-    __shared__ float sh_bcast[4];
+    __shared__ float sh_bcast[5];
 
     sa = warp_merge(sa, c);
     sb = warp_merge(sb, c);
@@ -107,19 +107,22 @@ __global__ void __launch_bounds__(K1_THREADS) row_stats_kernel(const VerifyParam
         rm = warp_argmax(rm);
         if (lane == 0) {
             sh_bcast[0] = ra.m; sh_bcast[1] = ra.s; sh_bcast[2] = rb.m; sh_bcast[3] = rb.s;
+            // q_v / p_v = 2^(yb - ya) sum_a / sum_b: the ratio of the sums folds into the draft row's offset
+            sh_bcast[4] = -rb.m * c + log2f(ra.s / rb.s);
             sh_am[0] = rm;
         }
     }
     __syncthreads();
     const float max_a = sh_bcast[0], sum_a = sh_bcast[1], max_b = sh_bcast[2], sum_b = sh_bcast[3];
 
-    // ---- sweep 2: sum_v min(p_v, q_v)
+    // ---- sweep 2: sum_v min(p_v, q_v) = (1 / sum_a) sum_v 2^min(ya_v, yb_v): one exponential per pair
     double total_min = 0.0;
     if (pair) {
-        const float nma = -max_a * c, nmb = -max_b * c;
-        const float ia = 1.0f / sum_a, ib = 1.0f / sum_b;
+        const float nma = -max_a * c, nmb = sh_bcast[4];
+        const float ia = 1.0f / sum_a;
         float acc = 0.f;
-        for (int i = tid; i < nvec; i += K1_THREADS) {
+        // backwards: the end of the rows was read last in sweep 1 and is the part most likely still in L2
+        for (int i = nvec - 1 - tid; i >= 0; i -= K1_THREADS) {
             float xa[VEC], xb[VEC];
             if constexpr (VECTOR) {
                 Logit<LT>::unpack(ld_stream(reinterpret_cast<const uint4 *>(a) + i), xa);
@@ -130,9 +133,9 @@ __global__ void __launch_bounds__(K1_THREADS) row_stats_kernel(const VerifyParam
             }
 #pragma unroll
             for (int e = 0; e < VEC; ++e)
-                acc += fminf(ex2(fmaf(xa[e], c, nma)) * ia, ex2(fmaf(xb[e], c, nmb)) * ib);
+                acc += ex2(fminf(fmaf(xa[e], c, nma), fmaf(xb[e], c, nmb)));
         }
-        double w = warp_sum((double)acc);
+        double w = warp_sum((double)(acc * ia));
         if (lane == 0) sh_min[warp] = w;
         __syncthreads();
         if (tid == 0) {
