@@ -22,6 +22,7 @@ struct metasd_ctx {
     float *stage_reward;
     bool fused_ready;
     FusedPlan plan;
+    int keep_permille;   // share of every row that the streaming kernel asks L2 to keep between its sweeps
     // split streaming path
     int grp_size, grp_ctas;
     GroupRecord *grp_rec;
@@ -117,6 +118,11 @@ int metasd_init(metasd_ctx **out, const metasd_config *cfg)
     if (!c) return METASD_ERR_NO_MEMORY;
     memset(c, 0, sizeof *c);
     c->cfg = *cfg;
+    {   // 650: the best measured value on B200 for 128k-152k vocabularies (METASD_KEEP_PERMILLE overrides, for tuning)
+        const char *kp = getenv("METASD_KEEP_PERMILLE");
+        const int v = kp && *kp ? atoi(kp) : 650;
+        c->keep_permille = v < 0 ? 0 : (v > 1000 ? 1000 : v);
+    }
     const size_t B = cfg->max_batch, K = cfg->n_drafters, tau = cfg->window, kp1 = cfg->max_draft + 1;
     cudaError_t e = cudaSuccess;
     auto alloc = [&](void **p, size_t bytes) {
@@ -225,6 +231,7 @@ int metasd_verify(metasd_ctx *ctx, int32_t batch, int32_t k, const void *target_
     p.seed = seed; p.beta = cfg.beta; p.gamma = cfg.gamma;
     p.accepted_len = accepted_len; p.next_token = next_token; p.reward = reward; p.diag = diag;
     p.st = ctx->st; p.stats = ctx->stats; p.status = ctx->status;
+    p.keep_permille = ctx->keep_permille;
     p.grp_size = ctx->grp_size; p.grp_ctas = ctx->grp_ctas;
     p.grp_rec = ctx->grp_rec; p.grp_min = ctx->grp_min; p.grp_count = ctx->grp_count;
     const size_t row_bytes = (size_t)cfg.vocab * logit_size(cfg.logit_dtype);

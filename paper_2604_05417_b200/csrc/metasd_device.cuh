@@ -94,6 +94,29 @@ __device__ __forceinline__ uint4 ld_stream(const void *p)
     return v;
 }
 
+// The same load with an L2 eviction policy (from createpolicy): evict_last keeps the line for a later re-read,
+// evict_first gives it up early.
+__device__ __forceinline__ uint64_t l2_policy_evict_last()
+{
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_first()
+{
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ uint4 ld_stream_hint(const void *p, uint64_t policy)
+{
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %5;"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p), "l"(policy));
+    return v;
+}
+
 // ---------------------------------------------------------------------------------------------
 // Online softmax statistics relative to the raw maximum m: s = sum 2^((x - m) c)
 // ---------------------------------------------------------------------------------------------

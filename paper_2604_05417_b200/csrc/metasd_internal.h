@@ -61,6 +61,7 @@ struct VerifyParams {
     RowStats *stats;   // [batch, k+1]
     uint32_t *status;
     int32_t vector_ok; // rows are 16-byte aligned and a whole number of 16-byte vectors
+    int32_t keep_permille;   // share of every row (its end) that the first sweep asks L2 to keep
     // split streaming path: grp_size CTAs share a row pair (0: one CTA per row pair)
     int32_t grp_size;
     int32_t grp_ctas;        // CTAs of the launch (co-resident)

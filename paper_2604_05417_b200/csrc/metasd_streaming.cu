@@ -49,11 +49,15 @@ __global__ void __launch_bounds__(K1_THREADS) row_stats_kernel(const VerifyParam
     // ---- sweep 1: online (max, sum) of both rows, arg-max of the target row
     MaxSum sa = {METASD_NEG_BIG, 0.f}, sb = {METASD_NEG_BIG, 0.f};
     ArgMax am = {METASD_NEG_BIG, 0x7FFFFFFF};
+    const uint64_t keep = l2_policy_evict_last(), drop = l2_policy_evict_first();
+    const int keep_from = nvec - (int)((long long)nvec * p.keep_permille / 1000);
     for (int i = tid; i < nvec; i += K1_THREADS) {
         float xa[VEC], xb[VEC];
         if constexpr (VECTOR) {
-            Logit<LT>::unpack(ld_stream(reinterpret_cast<const uint4 *>(a) + i), xa);
-            if (pair) Logit<LT>::unpack(ld_stream(reinterpret_cast<const uint4 *>(d) + i), xb);
+            // the end of the rows is asked to stay in L2 until the second sweep (which starts there) re-reads it
+            const uint64_t pol = i >= keep_from ? keep : drop;
+            Logit<LT>::unpack(ld_stream_hint(reinterpret_cast<const uint4 *>(a) + i, pol), xa);
+            if (pair) Logit<LT>::unpack(ld_stream_hint(reinterpret_cast<const uint4 *>(d) + i, pol), xb);
         } else {
             xa[0] = Logit<LT>::scalar(a, i);
             if (pair) xb[0] = Logit<LT>::scalar(d, i);
@@ -125,8 +129,8 @@ __global__ void __launch_bounds__(K1_THREADS) row_stats_kernel(const VerifyParam
         for (int i = nvec - 1 - tid; i >= 0; i -= K1_THREADS) {
             float xa[VEC], xb[VEC];
             if constexpr (VECTOR) {
-                Logit<LT>::unpack(ld_stream(reinterpret_cast<const uint4 *>(a) + i), xa);
-                Logit<LT>::unpack(ld_stream(reinterpret_cast<const uint4 *>(d) + i), xb);
+                Logit<LT>::unpack(ld_stream_hint(reinterpret_cast<const uint4 *>(a) + i, drop), xa);
+                Logit<LT>::unpack(ld_stream_hint(reinterpret_cast<const uint4 *>(d) + i, drop), xb);
             } else {
                 xa[0] = Logit<LT>::scalar(a, i);
                 xb[0] = Logit<LT>::scalar(d, i);
