@@ -59,14 +59,15 @@ def measured_peak_gbs():
         return 6650.0, "fallback"
 
 
+# DRAM bytes (read + write) of ONE launch of the dominant kernel, from the one-pass ncu capture of the full-size
+# launch that profiles/row_stats_kernel_cfg4.md summarises.  An entry is removed when its kernel changes.
+KNOWN_TRAFFIC = {
+    ("cfg4_greedy", "streaming"): 3.65e9 + 3.4e6,
+}
+
+
 def known_traffic(workload: str, path_name: str):
-    """DRAM bytes per launch of the dominant kernel from the committed ncu capture, if there is one."""
-    try:
-        with open(os.path.join(ROOT, "profiles", "dram_traffic.json")) as f:
-            table = json.load(f)
-        return table.get("%s/%s" % (workload, path_name))
-    except Exception:
-        return None
+    return KNOWN_TRAFFIC.get((workload, path_name))
 
 
 class ClockSampler:
@@ -237,7 +238,7 @@ def main():
     peak, peak_kind = measured_peak_gbs()
     achieved = bytes_round / (kernel_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": known_traffic(wl.name, path_name), "peak_kind": "of " + peak_kind,
+                "traffic": known_traffic(wl.name, path_name) if not args.batch else None, "peak_kind": "of " + peak_kind,
                 "algorithmic_bytes_per_launch": bytes_round, "kernel_ms": kernel_ms,
                 "frac_of_8TBs_nominal": achieved / 8000.0,
                 "note": "duration = CUDA events around select+verify of one step (%s path)" % path_name}
