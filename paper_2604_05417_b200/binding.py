@@ -20,7 +20,7 @@ BF16, FP32 = 0, 1
 UCB, DUCB, SWUCB = 0, 1, 2
 REWARD_BD, REWARD_BE = 0, 1
 PATH_AUTO, PATH_STREAMING, PATH_FUSED = 0, 1, 2
-STATUS_NONFINITE, STATUS_TOKEN_OOR, STATUS_Q_ZERO = 1, 2, 4
+STATUS_NONFINITE, STATUS_TOKEN_OOR, STATUS_Q_ZERO, STATUS_TIMEOUT, STATUS_BAD_POINTER = 1, 2, 4, 8, 16
 
 OK, ERR_INVALID_ARGUMENT, ERR_UNSUPPORTED, ERR_CUDA, ERR_NO_MEMORY, ERR_BAD_STATE_BLOB = 0, -1, -2, -3, -4, -5
 

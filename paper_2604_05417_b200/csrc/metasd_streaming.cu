@@ -25,7 +25,16 @@ template <typename LT>
 __device__ __forceinline__ const LT *draft_rows(const VerifyParams &p, int b)
 {
     if (p.draft) return reinterpret_cast<const LT *>(p.draft);
-    return reinterpret_cast<const LT *>(p.drafter_ptrs[p.st.arm[b]]);
+    const void *q = p.drafter_ptrs[p.st.arm[b]];
+    // A table entry that is NULL or not aligned like the target (16 bytes on the vector path) must never be
+    // dereferenced with vector loads: flag it and let the target's own rows stand in, so that the outputs of
+    // the sequence are defined (if meaningless) and nothing faults.
+    const uintptr_t mask = p.vector_ok ? 15u : (uintptr_t)(sizeof(LT) - 1);
+    if (q == nullptr || (reinterpret_cast<uintptr_t>(q) & mask) != 0) {
+        if (threadIdx.x == 0) atomicOr(p.status, METASD_STATUS_BAD_POINTER);
+        return reinterpret_cast<const LT *>(p.target);
+    }
+    return reinterpret_cast<const LT *>(q);
 }
 
 // -------------------------------------------------------------------------------------------

@@ -203,6 +203,29 @@ def test_reset_and_state_roundtrip(path):
         m.close()
 
 
+@pytest.mark.parametrize("path", PATHS)
+def test_misaligned_drafter_table_entry_is_flagged_not_dereferenced(path):
+    """A table pointer that is not 16-byte aligned sets a status bit; the rows behind it are never read."""
+    wl = base(B=4, N=2, k=3, V=1024, sigmas=(0.5, 2.0))
+    dev = torch.device("cuda", 0)
+    gen = RoundGenerator(wl, device=dev, seed=13)
+    from _harness import new_context
+    gpu = new_context(4, 2, 3, 1024, path=path)
+    rd = gen.table_round(0)
+    backing = torch.zeros(4 * 3 * 1024 + 8, dtype=torch.bfloat16, device=dev)
+    crooked = backing[1:1 + 4 * 3 * 1024].view(4, 3, 1024)          # starts 2 bytes past a 16-byte boundary
+    crooked.copy_(rd["drafts"][0])
+    assert crooked.data_ptr() % 16 == 2
+    table = M.pointer_table([crooked, rd["drafts"][1]])
+    for t in range(2):                                               # round 0 plays drafter 0 (the crooked one), round 1 drafter 1
+        res = gpu.verify(rd["target"], None, rd["tokens"], 1.0, 3, drafter_table=table, token_arm_stride=4 * 3)
+        torch.cuda.synchronize()
+        status = gpu.last_status()
+        assert bool(status & M.STATUS_BAD_POINTER) == (t == 0)
+        assert ((res.accepted_len >= 0) & (res.accepted_len <= 3)).all()
+    gpu.close()
+
+
 def test_argument_validation_on_device():
     gpu = M.MetaSD(2, 2, 3, 512)
     dev = torch.device("cuda", 0)
@@ -254,7 +277,7 @@ def test_verify_host_matches_device_call():
 
 
 @pytest.mark.parametrize("path", PATHS)
-@pytest.mark.parametrize("name", ["cfg4_greedy", "cfg3_tasks"])
+@pytest.mark.parametrize("name", ["cfg4_greedy", "cfg3_tasks", "cfg5_fp32_stress", "cfg2_nonstationary"])
 def test_full_size_launch_sampled_against_oracle(name, path):
     """The benchmark's launch configuration at full batch and vocabulary; the oracle re-computes a
     sample of sequences one by one (each keyed by its global sequence id)."""
