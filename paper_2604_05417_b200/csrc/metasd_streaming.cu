@@ -189,11 +189,9 @@ __device__ __forceinline__ uint32_t ld_acquire(const uint32_t *p)
     return v;
 }
 
-// Warp 0 of every CTA only communicates: while the other warps sweep, it publishes the CTA's record of one row
-// pair (fence + counter), waits (bounded) for the group's records of the row pair whose second sweep comes next,
-// merges them, and adds up and publishes the partial sums of min(p, q).  The global-memory round trips of the
-// exchange therefore overlap the sweeps.  The first sweep of the NEXT row pair runs before the second sweep of
-// the current one, so a group's records have a whole sweep's time to arrive.
+// Warp 0 of every CTA only communicates: it publishes the CTA's record of a row pair (a release increment, no
+// round trip), waits (bounded) for the group's records, merges them for the second sweep, and afterwards
+// publishes the CTA's partial sum of min(p, q); the CTAs of a group take turns in adding the parts up.
 template <typename LT>
 __global__ void __launch_bounds__(KS_THREADS, 3) split_row_stats_kernel(const VerifyParams p)
 {
@@ -207,6 +205,8 @@ __global__ void __launch_bounds__(KS_THREADS, 3) split_row_stats_kernel(const Ve
     const int n_groups = gridDim.x / G, grp = blockIdx.x / G, g = blockIdx.x - grp * G;
     const int nvec = V / VEC, per = (nvec + G - 1) / G;
     const int v_lo = min(g * per, nvec), v_hi = min(v_lo + per, nvec);   // this CTA's part of every row
+    const uint64_t keep = l2_policy_evict_last(), drop = l2_policy_evict_first();
+    const int keep_from = v_hi - (int)((long long)(v_hi - v_lo) * p.keep_permille / 1000);
     __shared__ MaxSum sh_a[NWARP], sh_b[NWARP];
     __shared__ ArgMax sh_am[NWARP];
     __shared__ double sh_min[NWARP];
@@ -229,8 +229,10 @@ __global__ void __launch_bounds__(KS_THREADS, 3) split_row_stats_kernel(const Ve
         ArgMax am = {METASD_NEG_BIG, 0x7FFFFFFF};
         for (int i = v_lo + st; i < v_hi; i += NSWEEP) {
             float xa[VEC], xb[VEC];
-            Logit<LT>::unpack(ld_stream(reinterpret_cast<const uint4 *>(a) + i), xa);
-            if (pair) Logit<LT>::unpack(ld_stream(reinterpret_cast<const uint4 *>(d) + i), xb);
+            // the end of this CTA's part is asked to stay in L2 until the second sweep (which starts there)
+            const uint64_t pol = i >= keep_from ? keep : drop;
+            Logit<LT>::unpack(ld_stream_hint(reinterpret_cast<const uint4 *>(a) + i, pol), xa);
+            if (pair) Logit<LT>::unpack(ld_stream_hint(reinterpret_cast<const uint4 *>(d) + i, pol), xb);
             float cm = xa[0];
 #pragma unroll
             for (int e = 1; e < VEC; ++e) cm = fmaxf(cm, xa[e]);
@@ -274,10 +276,10 @@ __global__ void __launch_bounds__(KS_THREADS, 3) split_row_stats_kernel(const Ve
         if (pair) {
             const float nma = -sh_bcast[0] * c, nmb = sh_bcast[4], sum_a = sh_bcast[1];
             float acc = 0.f;
-            for (int i = v_lo + st; i < v_hi; i += NSWEEP) {
+            for (int i = v_hi - 1 - st; i >= v_lo; i -= NSWEEP) {   // backwards: the end was read last
                 float xa[VEC], xb[VEC];
-                Logit<LT>::unpack(ld_stream(reinterpret_cast<const uint4 *>(a) + i), xa);
-                Logit<LT>::unpack(ld_stream(reinterpret_cast<const uint4 *>(d) + i), xb);
+                Logit<LT>::unpack(ld_stream_hint(reinterpret_cast<const uint4 *>(a) + i, drop), xa);
+                Logit<LT>::unpack(ld_stream_hint(reinterpret_cast<const uint4 *>(d) + i, drop), xb);
 #pragma unroll
                 for (int e = 0; e < VEC; ++e) acc += ex2(fminf(fmaf(xa[e], c, nma), fmaf(xb[e], c, nmb)));
             }
@@ -365,41 +367,26 @@ __global__ void __launch_bounds__(KS_THREADS, 3) split_row_stats_kernel(const Ve
         }
     };
 
-    // Group grp takes row pairs grp, grp + n_groups, ... in (sequence, position) order.
-    if (grp < n_items) {
-        if (warp != 0) first_sweep(grp);
-        __syncthreads();
-        if (warp == 0) publish_record(grp);
-    }
-    // warp 0: statistics of the row pair in its second sweep, and of the one before (for the finalising turn)
-    float m_a = 0.f, s_a = 0.f, m_b = 0.f, s_b = 0.f, pm_a = 0.f, ps_a = 0.f, pm_b = 0.f, ps_b = 0.f;
-    int arg = 0, parg = 0, prev = -1, turn = 0;
+    // Group grp takes row pairs grp, grp + n_groups, ... in (sequence, position) order: both sweeps of a row pair
+    // back to back (the second finds the first's bytes in L2), the group's exchange in between.
+    float m_a = 0.f, s_a = 0.f, m_b = 0.f, s_b = 0.f;
+    int arg = 0, turn = 0;
     for (int item = grp; item < n_items; item += n_groups, ++turn) {
-        const int next = item + n_groups;
-        // phase A: first sweep of the next row pair | warp 0 prepares the second sweep of this one
-        if (warp != 0) {
-            if (next < n_items) first_sweep(next);
-        } else {
+        if (warp != 0) first_sweep(item);
+        __syncthreads();
+        if (warp == 0) {
+            publish_record(item);
             merge_group(item);
             m_a = sh_bcast[0]; s_a = sh_bcast[1]; m_b = sh_bcast[2]; s_b = sh_bcast[3]; arg = sh_arg;
         }
         __syncthreads();
-        // phase B: second sweep of this row pair | warp 0 publishes the next one's record and, on its turn,
-        // writes the statistics of the previous row pair
-        if (warp != 0) {
-            second_sweep(item);
-        } else {
-            if (next < n_items) publish_record(next);
-            if (prev >= 0 && (turn - 1) % G == g) finalise(prev, pm_a, ps_a, pm_b, ps_b, parg);
-        }
+        if (warp != 0) second_sweep(item);
         __syncthreads();
-        // warp 0 publishes this row pair's partial sum while the others start the next phase A
         if (warp == 0) {
             publish_min(item);
-            prev = item; pm_a = m_a; ps_a = s_a; pm_b = m_b; ps_b = s_b; parg = arg;
+            if (turn % G == g) finalise(item, m_a, s_a, m_b, s_b, arg);   // the CTAs of a group take turns
         }
     }
-    if (warp == 0 && prev >= 0 && (turn - 1) % G == g) finalise(prev, pm_a, ps_a, pm_b, ps_b, parg);
 }
 
 // -------------------------------------------------------------------------------------------
