@@ -47,7 +47,14 @@ enum metasd_error {
 };
 
 enum metasd_dtype { METASD_BF16 = 0, METASD_FP32 = 1 };
-enum metasd_bandit { METASD_UCB = 0, METASD_DUCB = 1, METASD_SWUCB = 2 };
+enum metasd_bandit {
+    METASD_UCB = 0,   /* Algorithm 2 */
+    METASD_DUCB = 1,  /* Discounted UCB (non-stationary appendix) */
+    METASD_SWUCB = 2, /* Sliding-window UCB (non-stationary appendix) */
+    METASD_EXP3 = 3,  /* MetaSD-EXP3 (the algorithm box of that name): arms drawn from
+                         p_t(i) = (1 - gamma) w_i / sum w + gamma / K, w_a <- w_a exp(gamma (r / p_t(a)) / K) */
+    METASD_RAND = 4   /* the uniformly random baseline of the paper's tables */
+};
 enum metasd_reward { METASD_REWARD_BD = 0, METASD_REWARD_BE = 1 };
 
 /* Which kernels metasd_verify launches. */
@@ -68,8 +75,12 @@ enum metasd_path {
                                         outputs of the sequences that played that drafter are meaningless */
 
 /* Hyper-parameters of metasd_init.  Paper notation: n_drafters = K, max_draft = N_max, beta = the
- * exploration strength of Algorithm 2 (experiments: 0.01), gamma = the D-UCB decay, window = the
- * SW-UCB window tau (neither value is given in the paper; 0.975 / 50 are this library's defaults). */
+ * exploration strength of Algorithm 2 (experiments: 0.01), gamma = the D-UCB decay or, for METASD_EXP3, its
+ * mixing parameter (both are called gamma in the paper), window = the SW-UCB window tau (none of these values
+ * is given in the paper; 0.975 / 50 are this library's defaults).
+ * The randomised policies draw the arm of round t from word 2 of the Philox block keyed by the seed of the
+ * latest metasd_verify call (0 before the first one) at counter (sequence_base + b, t, 0xFFFFFFFF, 0):
+ * EXP3 by inverse CDF in arm order over the 24-bit uniform, RAND as floor(uniform * K). */
 typedef struct metasd_config {
     int32_t max_batch;          /* B: sequences, 1 .. 65535 */
     int32_t n_drafters;         /* K: 1 .. 16 */
@@ -114,7 +125,8 @@ int metasd_reset(metasd_ctx *ctx, const int32_t *seq_ids, int32_t n, void *strea
 
 /* Algorithm 2, lines 2-7: arm_out[b] = the drafter sequence b plays this round, b < batch.
  * Rounds t < K play arm t (the initial sweep); afterwards argmax_i mu_i + beta sqrt(2 ln t / n_i),
- * lowest index on ties; an arm with no pull inside the SW-UCB window scores +infinity. */
+ * lowest index on ties; an arm with no pull inside the SW-UCB window scores +infinity.  METASD_EXP3 and
+ * METASD_RAND: the arm drawn as described at metasd_config. */
 int metasd_select(metasd_ctx *ctx, int32_t batch, int32_t *arm_out, void *stream);
 
 /* One verification round for sequences 0 .. batch-1 (Algorithm 4 lines 6-12, Definition 2,

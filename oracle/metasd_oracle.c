@@ -32,6 +32,10 @@
 #define MSDO_UCB 0
 #define MSDO_DUCB 1
 #define MSDO_SWUCB 2
+#define MSDO_EXP3 3
+#define MSDO_RAND 4
+/* position index of the random-number block that draws a randomised policy's arm */
+#define MSDO_SELECT_POSITION 0xFFFFFFFFu
 
 #define MSDO_REWARD_BD 0
 #define MSDO_REWARD_BE 1
@@ -290,6 +294,8 @@ void msdo_verify_sequence(const double *target, const double *draft, const int32
 /*   stat_a[K], stat_b[K]                                                     */
 /*       UCB  : mu_hat_i, n_i                                                 */
 /*       D-UCB: discounted reward sum S_i, discounted count N_i               */
+/*       EXP3 : weights w_i, kept divided by their largest (stat_b unused)    */
+/*       Rand : nothing                                                       */
 /*   win_arm[tau], win_reward[tau] (SW-UCB): round s sits in slot s mod tau   */
 /* ------------------------------------------------------------------------- */
 
@@ -337,6 +343,41 @@ int msdo_bandit_select(int variant, int K, double beta, int tau, int t, const do
     return best;
 }
 
+/* MetaSD-EXP3 (the algorithm box "MetaSD-EXP3"): p_t(i) = (1 - gamma) w_i / sum_j w_j + gamma / K. */
+void msdo_exp3_probabilities(int K, double gamma, const double *w, double *prob)
+{
+    double sum = 0.0;
+    for (int i = 0; i < K; ++i) sum += w[i];
+    for (int i = 0; i < K; ++i) prob[i] = (1.0 - gamma) * (w[i] / sum) + gamma / (double)K;
+}
+
+/* The arm of round t for the randomised policies.  The uniform is word 2 of the Philox block
+ * (seed; sequence, t, MSDO_SELECT_POSITION, 0), 24 bits.
+ *   EXP3: inverse CDF over p_t(0..K-1) in arm order: the smallest i with sum_{j<=i} p_j > u (the last arm if
+ *         rounding leaves none).  gap: distance from u to the nearest CDF boundary.
+ *   Rand: arm = floor(u K), in integers: ((word >> 8) * K) >> 24.  gap: +infinity (nothing to round). */
+int msdo_random_select(int variant, int K, double gamma, int t, const double *stat_a, uint64_t seed,
+                       uint32_t sequence, double *gap)
+{
+    uint32_t ctr[4] = {sequence, (uint32_t)t, MSDO_SELECT_POSITION, 0u};
+    uint32_t key[2] = {(uint32_t)(seed & 0xFFFFFFFFu), (uint32_t)(seed >> 32)}, out[4];
+    msdo_philox4x32_10(ctr, key, out);
+    if (gap) *gap = INFINITY;
+    if (variant == MSDO_RAND) return (int)(((uint64_t)(out[2] >> 8) * (uint64_t)K) >> 24);
+    const double u = msdo_uniform24(out[2]);
+    double prob[64], cum = 0.0, nearest = INFINITY;
+    msdo_exp3_probabilities(K, gamma, stat_a, prob);
+    int arm = -1;
+    for (int i = 0; i < K; ++i) {
+        cum += prob[i];
+        if (i < K - 1 && fabs(u - cum) < nearest) nearest = fabs(u - cum);
+        if (arm < 0 && cum > u) arm = i;
+    }
+    if (arm < 0) arm = K - 1;
+    if (gap) *gap = nearest;
+    return arm;
+}
+
 /* The update after a round with arm a and reward r. */
 void msdo_bandit_update(int variant, int K, double gamma, int tau, int32_t *t, double *stat_a,
                         double *stat_b, int32_t *win_arm, double *win_reward, int a, double r)
@@ -350,6 +391,16 @@ void msdo_bandit_update(int variant, int K, double gamma, int tau, int32_t *t, d
         for (int i = 0; i < K; ++i) { stat_a[i] *= gamma; stat_b[i] *= gamma; }
         stat_a[a] += r;
         stat_b[a] += 1.0;
+    } else if (variant == MSDO_EXP3) {
+        /* r_hat = r / p_t(a); w_a <- w_a exp(gamma r_hat / K); the other weights stay.  The weights are then
+         * divided by their largest: the probabilities do not change and nothing overflows. */
+        double prob[64], top = 0.0;
+        msdo_exp3_probabilities(K, gamma, stat_a, prob);
+        stat_a[a] *= exp(gamma * (r / prob[a]) / (double)K);
+        for (int i = 0; i < K; ++i) if (stat_a[i] > top) top = stat_a[i];
+        for (int i = 0; i < K; ++i) stat_a[i] /= top;
+    } else if (variant == MSDO_RAND) {
+        /* no statistics */
     } else {
         win_arm[*t % tau] = a;
         win_reward[*t % tau] = r;
@@ -399,14 +450,19 @@ void msdo_verify_batch(int B, int k, int V, int dtype, const void *target, const
     }
 }
 
-void msdo_select_batch(int B, int variant, int K, double beta, int tau, const int32_t *t,
-                       const double *stat_a, const double *stat_b, const int32_t *win_arm,
-                       const double *win_reward, int32_t *arm, double *gap)
+void msdo_select_batch(int B, int variant, int K, double beta, double gamma, int tau, uint64_t seed,
+                       uint32_t sequence_base, const int32_t *t, const double *stat_a, const double *stat_b,
+                       const int32_t *win_arm, const double *win_reward, int32_t *arm, double *gap)
 {
-    for (int b = 0; b < B; ++b)
-        arm[b] = msdo_bandit_select(variant, K, beta, tau, t[b], stat_a + (size_t)b * K,
-                                    stat_b + (size_t)b * K, win_arm ? win_arm + (size_t)b * tau : NULL,
-                                    win_reward ? win_reward + (size_t)b * tau : NULL, gap ? gap + b : NULL);
+    for (int b = 0; b < B; ++b) {
+        if (variant == MSDO_EXP3 || variant == MSDO_RAND)
+            arm[b] = msdo_random_select(variant, K, gamma, t[b], stat_a + (size_t)b * K, seed,
+                                        sequence_base + (uint32_t)b, gap ? gap + b : NULL);
+        else
+            arm[b] = msdo_bandit_select(variant, K, beta, tau, t[b], stat_a + (size_t)b * K,
+                                        stat_b + (size_t)b * K, win_arm ? win_arm + (size_t)b * tau : NULL,
+                                        win_reward ? win_reward + (size_t)b * tau : NULL, gap ? gap + b : NULL);
+    }
 }
 
 void msdo_update_batch(int B, int variant, int K, double gamma, int tau, int32_t *t, double *stat_a,

@@ -21,7 +21,7 @@ _SRC = os.path.join(_HERE, "metasd_oracle.c")
 _LIB = os.path.join(_HERE, "libmetasd_oracle.so")
 
 DTYPE_BF16, DTYPE_FP32 = 0, 1
-UCB, DUCB, SWUCB = 0, 1, 2
+UCB, DUCB, SWUCB, EXP3, RAND = 0, 1, 2, 3, 4
 REWARD_BD, REWARD_BE = 0, 1
 STATUS_NONFINITE, STATUS_TOKEN_OOR, STATUS_Q_ZERO = 1, 2, 4
 
@@ -191,11 +191,14 @@ class OracleMetaSD:
         self.win_arm = np.zeros((B, tau), dtype=np.int32)
         self.win_reward = np.zeros((B, tau))
         self.last_gap = np.full(B, np.inf)
+        self.select_seed = 0            # key of a randomised policy's arm draw: 0 until the first verify call,
+        if cfg.bandit == EXP3:          # then the seed of the latest one
+            self.stat_a[:] = 1.0
 
     def reset(self, seq_ids=None):
         ids = slice(None) if seq_ids is None else np.asarray(seq_ids)
         self.t[ids] = 0
-        self.stat_a[ids] = 0
+        self.stat_a[ids] = 1.0 if self.cfg.bandit == EXP3 else 0.0      # EXP3: w_0(i) = 1
         self.stat_b[ids] = 0
         self.win_arm[ids] = 0
         self.win_reward[ids] = 0
@@ -206,7 +209,8 @@ class OracleMetaSD:
         arm = np.zeros(B, dtype=np.int32)
         gap = np.zeros(B)
         lib().msdo_select_batch(C.c_int(B), C.c_int(c.bandit), C.c_int(c.n_drafters),
-                                C.c_double(c.beta), C.c_int(max(c.tau, 1)), _p(self.t),
+                                C.c_double(c.beta), C.c_double(c.gamma), C.c_int(max(c.tau, 1)),
+                                C.c_uint64(self.select_seed), C.c_uint32(c.sequence_base), _p(self.t),
                                 _p(self.stat_a), _p(self.stat_b), _p(self.win_arm),
                                 _p(self.win_reward), _p(arm), _p(gap))
         self.last_gap[:B] = gap
@@ -253,6 +257,7 @@ class OracleMetaSD:
             _p(out["accept"]), _p(out["u_accept"]), _p(out["sample_margin"]), _p(out["status"]))
         if update:
             self.update(arm, out["reward"])
+            self.select_seed = seed
         out["next_arm"] = self.select(B) if update else None
         out["next_gap"] = self.last_gap[:B].copy()
         return out

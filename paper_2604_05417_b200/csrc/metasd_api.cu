@@ -56,7 +56,7 @@ int validate_config(const metasd_config *c)
     if (c->max_draft < 1 || c->max_draft > 16) return METASD_ERR_INVALID_ARGUMENT;
     if (c->vocab < 1) return METASD_ERR_INVALID_ARGUMENT;
     if (c->logit_dtype != METASD_BF16 && c->logit_dtype != METASD_FP32) return METASD_ERR_UNSUPPORTED;
-    if (c->bandit < METASD_UCB || c->bandit > METASD_SWUCB) return METASD_ERR_UNSUPPORTED;
+    if (c->bandit < METASD_UCB || c->bandit > METASD_RAND) return METASD_ERR_UNSUPPORTED;
     if (c->reward != METASD_REWARD_BD && c->reward != METASD_REWARD_BE) return METASD_ERR_UNSUPPORTED;
     if (c->path < METASD_PATH_AUTO || c->path > METASD_PATH_FUSED) return METASD_ERR_UNSUPPORTED;
     if (c->window < 1 || c->window > (1 << 20)) return METASD_ERR_INVALID_ARGUMENT;
@@ -154,7 +154,8 @@ int metasd_init(metasd_ctx **out, const metasd_config *cfg)
         }
     }
     if (e == cudaSuccess) e = cudaMemset(c->status, 0, sizeof(uint32_t));
-    if (e == cudaSuccess) e = launch_reset(c->st, cfg->max_batch, cfg->n_drafters, cfg->window, nullptr, cfg->max_batch, 0);
+    if (e == cudaSuccess) e = launch_reset(c->st, cfg->max_batch, cfg->n_drafters, cfg->window, cfg->bandit, cfg->gamma,
+                                            cfg->sequence_base, nullptr, cfg->max_batch, 0);
     if (e == cudaSuccess && cfg->path == METASD_PATH_FUSED &&
         fused_supported(cfg->logit_dtype, cfg->vocab, cfg->max_draft)) {
         e = fused_prepare(cfg->device, cfg->logit_dtype, cfg->vocab, cfg->max_batch, &c->plan);
@@ -183,7 +184,8 @@ int metasd_reset(metasd_ctx *ctx, const int32_t *seq_ids, int32_t n, void *strea
 {
     if (!ctx || n < 0) return METASD_ERR_INVALID_ARGUMENT;
     if (!seq_ids) n = ctx->cfg.max_batch;
-    CK(launch_reset(ctx->st, ctx->cfg.max_batch, ctx->cfg.n_drafters, ctx->cfg.window, seq_ids, n, (cudaStream_t)stream));
+    CK(launch_reset(ctx->st, ctx->cfg.max_batch, ctx->cfg.n_drafters, ctx->cfg.window, ctx->cfg.bandit, ctx->cfg.gamma,
+                    ctx->cfg.sequence_base, seq_ids, n, (cudaStream_t)stream));
     ctx->launches += n > 0;
     return METASD_OK;
 }

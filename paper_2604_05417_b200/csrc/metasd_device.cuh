@@ -176,10 +176,38 @@ __device__ __forceinline__ double warp_sum(double v)
 // ---------------------------------------------------------------------------------------------
 // Bandit arithmetic in fp64 (Algorithm 2; Discounted UCB; Sliding-window UCB)
 // ---------------------------------------------------------------------------------------------
-// Arm for round t of one sequence.  sa/sb: this sequence's [K] statistics; wa/wr: its window.
-__device__ inline int bandit_select(int variant, int K, double beta, int tau, int t, const double *sa,
-                                    const double *sb, const int32_t *wa, const double *wr)
+// Position index of the random-number block that draws a randomised policy's arm.
+#define METASD_SELECT_POSITION 0xFFFFFFFFu
+
+// MetaSD-EXP3: p_t(i) = (1 - gamma) w_i / sum_j w_j + gamma / K.
+__device__ inline double exp3_probability(int K, double gamma, const double *w, double sum, int i)
 {
+    return (1.0 - gamma) * (w[i] / sum) + gamma / (double)K;
+}
+
+// Arm of round t for the randomised policies: word 2 of the block (seed; sequence, t, METASD_SELECT_POSITION, 0).
+// EXP3: inverse CDF in arm order over the 24-bit uniform; RAND: floor(uniform * K) in integers.
+__device__ inline int random_select(int variant, int K, double gamma, int t, const double *w, uint64_t seed,
+                                    uint32_t sequence)
+{
+    const uint4 words = round_words(seed, sequence, (uint32_t)t, METASD_SELECT_POSITION);
+    if (variant == METASD_RAND) return (int)(((uint64_t)(words.z >> 8) * (uint64_t)K) >> 24);
+    const double u = (double)(words.z >> 8) * (1.0 / 16777216.0);
+    double sum = 0.0, cum = 0.0;
+    for (int i = 0; i < K; ++i) sum += w[i];
+    for (int i = 0; i < K; ++i) {
+        cum += exp3_probability(K, gamma, w, sum, i);
+        if (cum > u) return i;
+    }
+    return K - 1;
+}
+
+// Arm for round t of one sequence.  sa/sb: this sequence's [K] statistics; wa/wr: its window.
+__device__ inline int bandit_select(int variant, int K, double beta, double gamma, int tau, int t, const double *sa,
+                                    const double *sb, const int32_t *wa, const double *wr, uint64_t seed,
+                                    uint32_t sequence)
+{
+    if (variant == METASD_EXP3 || variant == METASD_RAND) return random_select(variant, K, gamma, t, sa, seed, sequence);
     if (t < K) return t;  // initial sweep: every drafter once, in order
     double mu[16], n[16];
     if (variant == METASD_SWUCB) {
@@ -220,6 +248,16 @@ __device__ inline void bandit_update(int variant, int K, double gamma, int tau, 
         for (int i = 0; i < K; ++i) { sa[i] *= gamma; sb[i] *= gamma; }
         sa[a] += r;
         sb[a] += 1.0;
+    } else if (variant == METASD_EXP3) {
+        // r_hat = r / p_t(a); w_a <- w_a exp(gamma r_hat / K); then all weights are divided by the largest one
+        // (the probabilities do not change and nothing overflows)
+        double sum = 0.0, top = 0.0;
+        for (int i = 0; i < K; ++i) sum += sa[i];
+        sa[a] *= exp(gamma * (r / exp3_probability(K, gamma, sa, sum, a)) / (double)K);
+        for (int i = 0; i < K; ++i) top = sa[i] > top ? sa[i] : top;
+        for (int i = 0; i < K; ++i) sa[i] /= top;
+    } else if (variant == METASD_RAND) {
+        // no statistics
     } else {
         int slot = *t % tau;
         wa[slot] = a;

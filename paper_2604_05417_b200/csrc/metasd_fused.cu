@@ -484,6 +484,16 @@ __device__ void warp_bandit(const VerifyParams &p, int b, int t, int arm, double
     double *sa = p.st.stat_a + (size_t)b * K, *sb = p.st.stat_b + (size_t)b * K;
     int32_t *wa = p.st.win_arm + (size_t)b * tau;
     double *wr = p.st.win_reward + (size_t)b * tau;
+    if (p.bandit == METASD_EXP3 || p.bandit == METASD_RAND) {   // a draw, not an arg-max: one lane does it
+        if (lane == 0) {
+            int32_t tt = t;
+            bandit_update(p.bandit, K, p.gamma, tau, &tt, sa, sb, wa, wr, arm, r);
+            p.st.t[b] = tt;
+            p.st.arm[b] = bandit_select(p.bandit, K, p.beta, p.gamma, tau, tt, sa, sb, wa, wr, p.seed,
+                                        p.sequence_base + (uint32_t)b);
+        }
+        return;
+    }
     double a_i = 0.0, b_i = 0.0;
     if (lane < K) { a_i = sa[lane]; b_i = sb[lane]; }
     if (p.bandit == METASD_UCB) {

@@ -93,7 +93,7 @@ cudaError_t launch_fused(const VerifyParams &p, int dtype, const FusedPlan &plan
 cudaError_t split_prepare(int device, int dtype, int V, int *resident_ctas, int *group_size);
 // small state kernels (metasd_streaming.cu)
 cudaError_t launch_select(const BanditState &st, int batch, int32_t *arm_out, cudaStream_t stream);
-cudaError_t launch_reset(const BanditState &st, int max_batch, int K, int tau, const int32_t *seq_ids,
-                         int n, cudaStream_t stream);
+cudaError_t launch_reset(const BanditState &st, int max_batch, int K, int tau, int variant, double gamma,
+                         uint32_t sequence_base, const int32_t *seq_ids, int n, cudaStream_t stream);
 
 }  // namespace metasd

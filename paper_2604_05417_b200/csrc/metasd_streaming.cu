@@ -624,7 +624,8 @@ __global__ void __launch_bounds__(K2_THREADS) epilogue_kernel(const VerifyParams
         int32_t *wa = p.st.win_arm + (size_t)b * p.tau;
         double *wr = p.st.win_reward + (size_t)b * p.tau;
         bandit_update(p.bandit, K, p.gamma, p.tau, &p.st.t[b], sa, sb, wa, wr, arm, r);
-        p.st.arm[b] = bandit_select(p.bandit, K, p.beta, p.tau, p.st.t[b], sa, sb, wa, wr);
+        p.st.arm[b] = bandit_select(p.bandit, K, p.beta, p.gamma, p.tau, p.st.t[b], sa, sb, wa, wr, p.seed,
+                                    p.sequence_base + (uint32_t)b);
         if (sh_flags) atomicOr(p.status, sh_flags);
     }
 }
@@ -705,20 +706,29 @@ __global__ void select_kernel(BanditState st, int batch, int32_t *arm_out)
     if (b < batch) arm_out[b] = st.arm[b];
 }
 
-__global__ void reset_kernel(BanditState st, int max_batch, int K, int tau, const int32_t *seq_ids, int n)
+__global__ void reset_kernel(BanditState st, int max_batch, int K, int tau, int variant, double gamma,
+                             uint32_t sequence_base, const int32_t *seq_ids, int n)
 {
     int i = blockIdx.x;
     if (i >= n) return;
     int b = seq_ids ? seq_ids[i] : i;
     if (b < 0 || b >= max_batch) return;
-    if (threadIdx.x == 0) { st.t[b] = 0; st.arm[b] = 0; }
+    const double first = variant == METASD_EXP3 ? 1.0 : 0.0;   // EXP3 starts from w(i) = 1
     for (int a = threadIdx.x; a < K; a += blockDim.x) {
-        st.stat_a[(size_t)b * K + a] = 0.0;
+        st.stat_a[(size_t)b * K + a] = first;
         st.stat_b[(size_t)b * K + a] = 0.0;
     }
     for (int s = threadIdx.x; s < tau; s += blockDim.x) {
         st.win_arm[(size_t)b * tau + s] = 0;
         st.win_reward[(size_t)b * tau + s] = 0.0;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        st.t[b] = 0;
+        // round 0: arm 0 of the initial sweep, or the randomised policies' draw (keyed by seed 0: no verify yet)
+        st.arm[b] = bandit_select(variant, K, 0.0, gamma, tau, 0, st.stat_a + (size_t)b * K, st.stat_b + (size_t)b * K,
+                                  st.win_arm + (size_t)b * tau, st.win_reward + (size_t)b * tau, 0ull,
+                                  sequence_base + (uint32_t)b);
     }
 }
 
@@ -728,11 +738,11 @@ cudaError_t launch_select(const BanditState &st, int batch, int32_t *arm_out, cu
     return cudaGetLastError();
 }
 
-cudaError_t launch_reset(const BanditState &st, int max_batch, int K, int tau, const int32_t *seq_ids, int n,
-                         cudaStream_t stream)
+cudaError_t launch_reset(const BanditState &st, int max_batch, int K, int tau, int variant, double gamma,
+                         uint32_t sequence_base, const int32_t *seq_ids, int n, cudaStream_t stream)
 {
     if (n <= 0) return cudaSuccess;
-    reset_kernel<<<n, 64, 0, stream>>>(st, max_batch, K, tau, seq_ids, n);
+    reset_kernel<<<n, 64, 0, stream>>>(st, max_batch, K, tau, variant, gamma, sequence_base, seq_ids, n);
     return cudaGetLastError();
 }
 

@@ -91,6 +91,16 @@ def test_cfg5_fp32_scaled(path, bandit):
 
 
 @pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("bandit", ["exp3", "rand"])
+def test_randomised_policies(path, bandit):
+    """MetaSD-EXP3 and the uniformly random baseline: arm draws, weights and round counters follow the oracle."""
+    from _harness import run_lockstep
+    wl = base(B=9, N=4, k=3, V=2048, sigmas=(0.3, 1.0, 2.0, 3.5)).scaled(gamma=0.2)
+    c = report(run_lockstep(wl, rounds=40, path=path, bandit=bandit, table_mode=True))
+    assert c["rounds"] == 40
+
+
+@pytest.mark.parametrize("path", PATHS)
 def test_pointer_table_mode(path):
     """The kernel indexes a table of K drafter tensors and a [K,B,k] token table by arm."""
     from _harness import run_lockstep

@@ -190,3 +190,126 @@ def test_first_selection_after_the_sweep_uses_ln_of_completed_rounds():
     assert O.bandit_select(O.UCB, 2, 1.14, 1, 3, mu, n)[0] == 0
     assert O.bandit_select(O.UCB, 2, 1.16, 1, 3, mu, n)[0] == 1
     assert O.bandit_select(O.UCB, 2, 1.40, 1, 3, mu, n)[0] == 1
+
+
+# ---------------------------------------------------------------------------------------------
+# MetaSD-EXP3 and the uniformly random baseline (the algorithm box "MetaSD-EXP3"; "Rand" in the tables)
+# ---------------------------------------------------------------------------------------------
+SELECT_POSITION = 0xFFFFFFFF
+
+
+def select_uniform(seed, sequence, t):
+    """The 24-bit uniform that draws a randomised policy's arm: word 2 of the block (sequence, t, 0xFFFFFFFF, 0)."""
+    w = O.philox4x32_10((sequence, t, SELECT_POSITION, 0), (seed & 0xFFFFFFFF, seed >> 32))
+    return (w[2] >> 8) / float(1 << 24), w[2]
+
+
+def exp3_probabilities(w, gamma):
+    w = np.asarray(w, dtype=np.float64)
+    return (1.0 - gamma) * w / w.sum() + gamma / len(w)
+
+
+def test_exp3_one_round_by_hand():
+    """K = 2, gamma = 1/2, first round: p = (1/2, 1/2); reward r on arm a gives w_a = exp(gamma r / (K p_a)) = exp(r / 2)."""
+    o = O.OracleMetaSD(O.OracleConfig(max_batch=1, n_drafters=2, vocab=4, bandit=O.EXP3, gamma=0.5))
+    a = int(o.select()[0])
+    o.update(np.array([a]), np.array([0.8]))
+    w = o.stat_a[0]
+    assert w.max() == 1.0                                        # kept divided by the largest weight
+    ratio = w[a] / w[1 - a]
+    assert abs(ratio - np.exp(0.4)) < 1e-14
+    p = exp3_probabilities([np.exp(0.4), 1.0] if a == 0 else [1.0, np.exp(0.4)], 0.5)
+    assert abs(p[a] - (0.5 * np.exp(0.4) / (np.exp(0.4) + 1.0) + 0.25)) < 1e-15
+    assert o.t[0] == 1
+
+
+def test_exp3_weights_follow_the_closed_form_of_the_importance_weighted_sums():
+    """log(w_j / w_i) = (gamma / K) (sum_t r_hat_j - sum_t r_hat_i), with r_hat = r / p_t(a_t) on the played arm."""
+    K, gamma, T = 4, 0.2, 300
+    o = O.OracleMetaSD(O.OracleConfig(max_batch=1, n_drafters=K, vocab=4, bandit=O.EXP3, gamma=gamma))
+    rng = np.random.RandomState(5)
+    sums = np.zeros(K)
+    w_ref = np.ones(K)
+    for t in range(T):
+        a = int(o.select()[0])
+        p = exp3_probabilities(w_ref, gamma)
+        r = float(rng.uniform(0.0, 1.0)) * (0.9 if a == 1 else 0.4)
+        sums[a] += r / p[a]
+        w_ref = np.exp(gamma / K * (sums - sums.max()))
+        o.update(np.array([a]), np.array([r]))
+        assert np.allclose(o.stat_a[0], w_ref, rtol=1e-11, atol=0)
+    assert sums.argmax() == 1                                     # the arm with the larger rewards collects the weight
+
+
+def test_exp3_draw_is_the_inverse_cdf_of_its_probabilities_on_the_documented_uniform():
+    K, gamma = 5, 0.3
+    B = 400
+    o = O.OracleMetaSD(O.OracleConfig(max_batch=B, n_drafters=K, vocab=4, bandit=O.EXP3, gamma=gamma, sequence_base=11))
+    rng = np.random.RandomState(2)
+    o.stat_a[:] = rng.uniform(0.05, 1.0, size=(B, K))
+    o.t[:] = rng.randint(0, 50, size=B)
+    o.select_seed = 0x1234567890
+    arm = o.select()
+    for b in range(B):
+        u, _ = select_uniform(0x1234567890, 11 + b, int(o.t[b]))
+        cdf = np.cumsum(exp3_probabilities(o.stat_a[b], gamma))
+        assert arm[b] == min(int(np.searchsorted(cdf, u, side="right")), K - 1)      # smallest i with cdf_i > u
+        edges = np.abs(u - cdf[:-1])
+        assert abs(o.last_gap[b] - edges.min()) < 1e-15
+
+
+def test_exp3_with_gamma_one_is_uniform_whatever_the_rewards():
+    K, B, T = 4, 64, 200
+    o = O.OracleMetaSD(O.OracleConfig(max_batch=B, n_drafters=K, vocab=4, bandit=O.EXP3, gamma=1.0))
+    counts = np.zeros(K)
+    for t in range(T):
+        a = o.select()
+        counts += np.bincount(a, minlength=K)
+        o.update(a, np.where(a == 0, 1.0, 0.0))                  # arm 0 always wins: irrelevant at gamma = 1
+        o.select_seed = t + 1
+    chi2 = ((counts - B * T / K) ** 2 / (B * T / K)).sum()
+    assert chi2 < 16.27                                          # chi-square, 3 degrees of freedom, p = 0.001
+
+
+def test_exp3_selection_frequencies_match_its_probabilities():
+    K, gamma, B = 3, 0.2, 30000
+    o = O.OracleMetaSD(O.OracleConfig(max_batch=B, n_drafters=K, vocab=4, bandit=O.EXP3, gamma=gamma))
+    o.stat_a[:] = np.array([1.0, 0.25, 0.5])
+    o.select_seed = 99
+    counts = np.bincount(o.select(), minlength=K)
+    expect = B * exp3_probabilities([1.0, 0.25, 0.5], gamma)
+    assert (((counts - expect) ** 2) / expect).sum() < 13.82     # chi-square, 2 degrees of freedom, p = 0.001
+
+
+def test_exp3_gain_respects_the_bound_of_its_source():
+    """Auer et al. (2002), Theorem 3.1: G_max - E[G_EXP3] <= (e - 1) gamma G_max + K ln K / gamma."""
+    K, gamma, T, B = 3, 0.15, 600, 64
+    means = np.array([0.2, 0.8, 0.5])
+    o = O.OracleMetaSD(O.OracleConfig(max_batch=B, n_drafters=K, vocab=4, bandit=O.EXP3, gamma=gamma))
+    rng = np.random.RandomState(3)
+    gain = np.zeros(B)
+    for t in range(T):
+        a = o.select()
+        r = np.clip(means[a] + rng.uniform(-0.1, 0.1, size=B), 0.0, 1.0)
+        gain += r
+        o.update(a, r)
+        o.select_seed = 1000 + t
+    g_max = means.max() * T
+    assert gain.mean() >= g_max - ((np.e - 1.0) * gamma * g_max + K * np.log(K) / gamma)
+    assert gain.mean() > means.mean() * T + 0.15 * T * (means.max() - means.mean())   # and it does learn
+
+
+def test_rand_is_floor_of_u_times_k_in_integers_and_uniform():
+    K, B = 7, 21000
+    o = O.OracleMetaSD(O.OracleConfig(max_batch=B, n_drafters=K, vocab=4, bandit=O.RAND, sequence_base=3))
+    o.t[:] = np.arange(B) % 17
+    o.select_seed = 42
+    arm = o.select()
+    for b in range(0, B, 97):
+        _, word = select_uniform(42, 3 + b, int(o.t[b]))
+        assert arm[b] == ((word >> 8) * K) >> 24
+    counts = np.bincount(arm, minlength=K)
+    assert (((counts - B / K) ** 2) / (B / K)).sum() < 22.46     # chi-square, 6 degrees of freedom, p = 0.001
+    before = o.stat_a.copy()
+    o.update(arm, np.ones(B))
+    assert np.array_equal(o.stat_a, before) and (o.t == np.arange(B) % 17 + 1).all()   # no statistics, t advances
