@@ -71,8 +71,8 @@ enum metasd_path {
 #define METASD_STATUS_TOKEN_OOR 2u /* a drafted token id was outside [0, V) */
 #define METASD_STATUS_Q_ZERO    4u /* the drafter gave probability 0 to its own drafted token */
 #define METASD_STATUS_TIMEOUT   8u /* a bounded wait on an asynchronous copy ran out: outputs of that call are undefined */
-#define METASD_STATUS_BAD_POINTER 16u /* a drafter-table entry was NULL or misaligned: its rows were not read and the
-                                        outputs of the sequences that played that drafter are meaningless */
+#define METASD_STATUS_BAD_POINTER 16u /* the drafter table of a call held a NULL or misaligned entry: its rows are never
+                                        read and the outputs of the sequences that played that drafter are meaningless */
 
 /* Hyper-parameters of metasd_init.  Paper notation: n_drafters = K, max_draft = N_max, beta = the
  * exploration strength of Algorithm 2 (experiments: 0.01), gamma = the D-UCB decay or, for METASD_EXP3, its

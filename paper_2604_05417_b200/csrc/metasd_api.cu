@@ -15,6 +15,7 @@ struct metasd_ctx {
     BanditState st;
     RowStats *stats;     // scratch of the streaming path: [max_batch, max_draft + 1]
     uint32_t *status;    // device status word
+    const void **table_clean;   // the checked copy of the caller's drafter table (16 entries)
     uint64_t launches;
     // staging for metasd_verify_host
     void *stage_target, *stage_draft;
@@ -136,6 +137,7 @@ int metasd_init(metasd_ctx **out, const metasd_config *cfg)
     alloc((void **)&c->st.win_reward, B * tau * sizeof(double));
     alloc((void **)&c->stats, B * kp1 * sizeof(RowStats));
     alloc((void **)&c->status, sizeof(uint32_t));
+    alloc((void **)&c->table_clean, 16 * sizeof(void *));
     if (cfg->host_staging) {
         const size_t row = (size_t)cfg->vocab * logit_size(cfg->logit_dtype);
         alloc(&c->stage_target, B * kp1 * row);
@@ -243,6 +245,14 @@ int metasd_verify(metasd_ctx *ctx, int32_t batch, int32_t k, const void *target_
                   (draft_logits ? ((uintptr_t)draft_logits % 16) == 0 : 1);
 
     cudaError_t e;
+    if (drafter_ptrs && metasd_resolved_path(ctx, k) != METASD_PATH_FUSED) {   // the fused kernel checks for itself
+        const uint32_t mask = p.vector_ok ? 15u : (uint32_t)(logit_size(cfg.logit_dtype) - 1);
+        e = launch_sanitize_table(drafter_ptrs, cfg.n_drafters, target_logits, mask, ctx->table_clean, ctx->status,
+                                  (cudaStream_t)stream);
+        if (e != cudaSuccess) return cuda_fail(e);
+        ctx->launches += 1;
+        p.drafter_ptrs = ctx->table_clean;
+    }
     if (metasd_resolved_path(ctx, k) == METASD_PATH_FUSED && p.vector_ok)
         e = launch_fused(p, cfg.logit_dtype, ctx->plan, (cudaStream_t)stream, &ctx->launches);
     else if (cfg.path == METASD_PATH_FUSED)

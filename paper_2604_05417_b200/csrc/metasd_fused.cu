@@ -582,7 +582,13 @@ __global__ void __launch_bounds__(FUSED_MAX_THREADS, 2) fused_round_kernel(const
         sh.token = -1;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (tid < 16) sh.table[tid] = (p.drafter_ptrs && tid < p.K) ? p.drafter_ptrs[tid] : nullptr;
+    if (tid < 16) {
+        const void *q = (p.drafter_ptrs && tid < p.K) ? p.drafter_ptrs[tid] : nullptr;
+        sh.table[tid] = q;
+        // a table entry that must not be read (NULL, misaligned) is flagged once per call, played or not
+        if (p.drafter_ptrs && tid < p.K && blockIdx.x == 0 && (q == nullptr || (reinterpret_cast<uintptr_t>(q) & 15u) != 0))
+            atomicOr(p.status, METASD_STATUS_BAD_POINTER);
+    }
     cluster_sync_all();   // every CTA of the cluster is running, its barriers initialised, before a peer writes to it
 
     // ---- producer (thread 0): one item = the chunks of a target slice and, below the bonus position, of a draft slice

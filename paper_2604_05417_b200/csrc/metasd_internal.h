@@ -91,6 +91,9 @@ cudaError_t launch_fused(const VerifyParams &p, int dtype, const FusedPlan &plan
 // how many CTAs of the split kernel are co-resident, and how many of them should share a row pair so that
 // the rows in flight stay inside L2 (1: not worth splitting)
 cudaError_t split_prepare(int device, int dtype, int V, int *resident_ctas, int *group_size);
+// copies the drafter table, flagging and replacing entries that must not be dereferenced (metasd_streaming.cu)
+cudaError_t launch_sanitize_table(const void *const *table, int K, const void *target, uint32_t mask, const void **clean,
+                                  uint32_t *status, cudaStream_t stream);
 // small state kernels (metasd_streaming.cu)
 cudaError_t launch_select(const BanditState &st, int batch, int32_t *arm_out, cudaStream_t stream);
 cudaError_t launch_reset(const BanditState &st, int max_batch, int K, int tau, int variant, double gamma,

@@ -19,22 +19,12 @@
 namespace metasd {
 
 constexpr int K1_THREADS = 512;
-constexpr int K2_THREADS = 256;
 
 template <typename LT>
 __device__ __forceinline__ const LT *draft_rows(const VerifyParams &p, int b)
 {
     if (p.draft) return reinterpret_cast<const LT *>(p.draft);
-    const void *q = p.drafter_ptrs[p.st.arm[b]];
-    // A table entry that is NULL or not aligned like the target (16 bytes on the vector path) must never be
-    // dereferenced with vector loads: flag it and let the target's own rows stand in, so that the outputs of
-    // the sequence are defined (if meaningless) and nothing faults.
-    const uintptr_t mask = p.vector_ok ? 15u : (uintptr_t)(sizeof(LT) - 1);
-    if (q == nullptr || (reinterpret_cast<uintptr_t>(q) & mask) != 0) {
-        if (threadIdx.x == 0) atomicOr(p.status, METASD_STATUS_BAD_POINTER);
-        return reinterpret_cast<const LT *>(p.target);
-    }
-    return reinterpret_cast<const LT *>(q);
+    return reinterpret_cast<const LT *>(p.drafter_ptrs[p.st.arm[b]]);   // the table was checked by sanitize_table_kernel
 }
 
 // -------------------------------------------------------------------------------------------
@@ -419,7 +409,7 @@ __device__ __forceinline__ void draw_weights(const LT *a, const LT *d, int i, in
 
 // Inverse CDF in token order over one row (pair): the smallest v with sum_{w<=v} weight_w > u * total.
 // Every warp owns a contiguous range of vectors; totals and offsets are carried in fp64.
-template <typename LT, bool VECTOR>
+template <typename LT, bool VECTOR, int K2_THREADS>
 __device__ int block_inverse_cdf(const LT *a, const LT *d, int V, int mode, float u, float c, float max_a,
                                  float sum_a, float max_b, float sum_b, double *sh_tot, int *sh_tok)
 {
@@ -515,7 +505,9 @@ __device__ int block_inverse_cdf(const LT *a, const LT *d, int V, int mode, floa
     return *sh_tok;
 }
 
-template <typename LT, bool VECTOR>
+// K2_THREADS: the draw walks one row pair per sequence, so a small batch wants large CTAs (many warps keep the
+// load chains short) and a large batch wants many small ones.
+template <typename LT, bool VECTOR, int K2_THREADS>
 __global__ void __launch_bounds__(K2_THREADS) epilogue_kernel(const VerifyParams p)
 {
     const int b = blockIdx.x, tid = threadIdx.x;
@@ -608,10 +600,10 @@ __global__ void __launch_bounds__(K2_THREADS) epilogue_kernel(const VerifyParams
         const RowStats rs = stats[n_acc];
         const LT *a = target + (size_t)n_acc * V;
         const LT *d = mode == 1 ? draft + (size_t)n_acc * V : nullptr;
-        token = block_inverse_cdf<LT, VECTOR>(a, d, V, mode, sh_u, c, rs.max_a, rs.sum_a, rs.max_b, rs.sum_b,
+        token = block_inverse_cdf<LT, VECTOR, K2_THREADS>(a, d, V, mode, sh_u, c, rs.max_a, rs.sum_a, rs.max_b, rs.sum_b,
                                               sh_tot, &sh_tok);
         if (token < 0 && mode == 1)  // p == q in fp32 yet rejected: draw from p
-            token = block_inverse_cdf<LT, VECTOR>(a, nullptr, V, 2, sh_u, c, rs.max_a, rs.sum_a, rs.max_b,
+            token = block_inverse_cdf<LT, VECTOR, K2_THREADS>(a, nullptr, V, 2, sh_u, c, rs.max_a, rs.sum_a, rs.max_b,
                                                   rs.sum_b, sh_tot, &sh_tok);
     }
 
@@ -637,6 +629,7 @@ template <typename LT>
 static cudaError_t launch_streaming_t(const VerifyParams &p, cudaStream_t stream, uint64_t *launches)
 {
     dim3 g1(p.k + 1, p.batch), g2(p.batch);
+    const bool big_ctas = p.batch <= 320;   // up to about two sequences per SM
     if (p.vector_ok && p.grp_size > 1) {
         const int n_items = p.batch * (p.k + 1);
         int n_groups = p.grp_ctas / p.grp_size;
@@ -649,13 +642,16 @@ static cudaError_t launch_streaming_t(const VerifyParams &p, cudaStream_t stream
         e = cudaLaunchCooperativeKernel(reinterpret_cast<const void *>(&split_row_stats_kernel<LT>), dim3(n_groups * p.grp_size),
                                         dim3(KS_THREADS), args, 0, stream);
         if (e != cudaSuccess) return e;
-        epilogue_kernel<LT, true><<<g2, K2_THREADS, 0, stream>>>(p);
     } else if (p.vector_ok) {
         row_stats_kernel<LT, true><<<g1, K1_THREADS, 0, stream>>>(p);
-        epilogue_kernel<LT, true><<<g2, K2_THREADS, 0, stream>>>(p);
     } else {
         row_stats_kernel<LT, false><<<g1, K1_THREADS, 0, stream>>>(p);
-        epilogue_kernel<LT, false><<<g2, K2_THREADS, 0, stream>>>(p);
+    }
+    if (p.vector_ok) {
+        if (big_ctas) epilogue_kernel<LT, true, 512><<<g2, 512, 0, stream>>>(p);
+        else epilogue_kernel<LT, true, 256><<<g2, 256, 0, stream>>>(p);
+    } else {
+        epilogue_kernel<LT, false, 256><<<g2, 256, 0, stream>>>(p);
     }
     *launches += 2;
     return cudaGetLastError();
@@ -695,6 +691,33 @@ cudaError_t split_prepare(int device, int dtype, int V, int *resident_ctas, int 
     *resident_ctas = resident - resident % G;
     *group_size = G;
     return cudaSuccess;
+}
+
+// -------------------------------------------------------------------------------------------
+// drafter table check
+// -------------------------------------------------------------------------------------------
+// Copies the caller's table of K drafter pointers into the context's own table.  An entry that is NULL or not
+// aligned like the target (16 bytes on the vector path, else the element size) must never be dereferenced: it is
+// flagged and replaced by the target pointer, so that the outputs of the sequences that play that drafter are
+// defined (if meaningless) and nothing faults.
+__global__ void sanitize_table_kernel(const void *const *table, int K, const void *target, uint32_t mask,
+                                      const void **clean, uint32_t *status)
+{
+    const int i = threadIdx.x;
+    if (i >= K) return;
+    const void *q = table[i];
+    if (q == nullptr || (reinterpret_cast<uintptr_t>(q) & mask) != 0) {
+        atomicOr(status, METASD_STATUS_BAD_POINTER);
+        q = target;
+    }
+    clean[i] = q;
+}
+
+cudaError_t launch_sanitize_table(const void *const *table, int K, const void *target, uint32_t mask, const void **clean,
+                                  uint32_t *status, cudaStream_t stream)
+{
+    sanitize_table_kernel<<<1, 32, 0, stream>>>(table, K, target, mask, clean, status);
+    return cudaGetLastError();
 }
 
 // -------------------------------------------------------------------------------------------

@@ -231,7 +231,7 @@ def test_misaligned_drafter_table_entry_is_flagged_not_dereferenced(path):
         res = gpu.verify(rd["target"], None, rd["tokens"], 1.0, 3, drafter_table=table, token_arm_stride=4 * 3)
         torch.cuda.synchronize()
         status = gpu.last_status()
-        assert bool(status & M.STATUS_BAD_POINTER) == (t == 0)
+        assert status & M.STATUS_BAD_POINTER                         # flagged on every call that is handed this table
         assert ((res.accepted_len >= 0) & (res.accepted_len <= 3)).all()
     gpu.close()
 
