@@ -411,18 +411,19 @@ __device__ __forceinline__ void draw_weights(const LT *a, const LT *d, int i, in
 // Every warp owns a contiguous range of vectors; totals and offsets are carried in fp64.
 template <typename LT, bool VECTOR, int K2_THREADS>
 __device__ int block_inverse_cdf(const LT *a, const LT *d, int V, int mode, float u, float c, float max_a,
-                                 float sum_a, float max_b, float sum_b, double *sh_tot, int *sh_tok)
+                                 float sum_a, float max_b, float sum_b, double *sh_tot, double *sh_sub, int *sh_tok,
+                                 int rank, int csize)
 {
     constexpr int VEC = VECTOR ? Logit<LT>::VEC : 1;
     constexpr int NWARP = K2_THREADS / 32;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int nvec = V / VEC;
-    const int per_warp = (nvec + NWARP - 1) / NWARP;
-    const int v0 = min(warp * per_warp, nvec), v1 = min(v0 + per_warp, nvec);
+    const int nwt = NWARP * csize, gw = rank * NWARP + warp;   // warps of the whole cluster, this warp among them
+    const int per_warp = (nvec + nwt - 1) / nwt;
+    const int v0 = min(gw * per_warp, nvec), v1 = min(v0 + per_warp, nvec);
     const float nma = -max_a * c, nmb = -max_b * c;
     const float ia = 1.0f / sum_a, ib = 1.0f / sum_b;
 
-    __syncthreads();  // the shared slots may still be read from an earlier call
     double acc = 0.0;
     for (int i = v0 + lane; i < v1; i += 32) {
         float w[VEC];
@@ -433,23 +434,59 @@ __device__ int block_inverse_cdf(const LT *a, const LT *d, int V, int mode, floa
         acc += (double)s;
     }
     acc = warp_sum(acc);
-    if (lane == 0) sh_tot[warp] = acc;
+    // Every CTA of the cluster is running (a peer's shared memory may not be written before that) and has
+    // finished reading the slots of an earlier call.
+    cluster_sync_all();
+    // every CTA of the cluster gets every warp's total
+    if (lane < csize) st_cluster(map_to_rank(smem_addr(&sh_tot[gw]), (uint32_t)lane), acc);
     if (tid == 0) *sh_tok = -1;
-    __syncthreads();
+    cluster_sync_all();
     double total = 0.0;
-    for (int w = 0; w < NWARP; ++w) total += sh_tot[w];
-    if (!(total > 0.0)) { __syncthreads(); return -1; }
+    for (int w = 0; w < nwt; ++w) total += sh_tot[w];
+    if (!(total > 0.0)) { cluster_sync_all(); return -1; }
     const double threshold = (double)u * total;
     // the warp whose range holds the crossing; rounding may leave none: then the last warp with mass
     int wstar = -1, wlast = -1;
     double base = 0.0, run = 0.0, base_last = 0.0;
-    for (int w = 0; w < NWARP; ++w) {
+    for (int w = 0; w < nwt; ++w) {
         if (sh_tot[w] > 0.0) { wlast = w; base_last = run; }
         if (wstar < 0 && run + sh_tot[w] > threshold) { wstar = w; base = run; }
         run += sh_tot[w];
     }
     if (wstar < 0) { wstar = wlast; base = base_last; }
-    if (warp == wstar) {
+    // second level, in the CTA that owns that range: each of its warps takes a part of it, so that the final scan
+    // is a trip or two instead of a long chain of dependent loads in one warp
+    if (rank == wstar / NWARP) {
+    const int r0 = min(wstar * per_warp, nvec), r1 = min(r0 + per_warp, nvec);
+    const int per_sub = (r1 - r0 + NWARP - 1) / NWARP;
+    const int s0 = min(r0 + warp * per_sub, r1), s1 = min(s0 + per_sub, r1);
+    {
+        double acc2 = 0.0;
+        for (int i = s0 + lane; i < s1; i += 32) {
+            float w[VEC];
+            draw_weights<LT, VEC>(a, d, i, mode, c, nma, ia, nmb, ib, w);
+            float s = 0.f;
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) s += w[e];
+            acc2 += (double)s;
+        }
+        acc2 = warp_sum(acc2);
+        if (lane == 0) sh_sub[warp] = acc2;
+    }
+    __syncthreads();
+    int sstar = -1, slast = -1;
+    {
+        double run2 = base, base2 = base, base2_last = base;
+        for (int w = 0; w < NWARP; ++w) {
+            if (sh_sub[w] > 0.0) { slast = w; base2_last = run2; }
+            if (sstar < 0 && run2 + sh_sub[w] > threshold) { sstar = w; base2 = run2; }
+            run2 += sh_sub[w];
+        }
+        if (sstar < 0) { sstar = slast; base2 = base2_last; }
+        base = base2;
+    }
+    if (warp == sstar) {
+        const int v0 = s0, v1 = s1;
         int found = -1, last_pos = -1;
         double run_base = base;
         for (int i0 = v0; i0 < v1 && found < 0; i0 += 32) {
@@ -499,9 +536,11 @@ __device__ int block_inverse_cdf(const LT *a, const LT *d, int V, int mode, floa
             for (int o = 16; o > 0; o >>= 1) last_pos = max(last_pos, __shfl_xor_sync(0xFFFFFFFFu, last_pos, o));
             found = last_pos;
         }
-        if (lane == 0) *sh_tok = found;
+        // every CTA of the cluster gets the token: they must all agree on whether the draw found one
+        if (lane < csize) st_cluster(map_to_rank(smem_addr(sh_tok), (uint32_t)lane), (int32_t)found);
     }
-    __syncthreads();
+    }
+    cluster_sync_all();
     return *sh_tok;
 }
 
@@ -510,7 +549,10 @@ __device__ int block_inverse_cdf(const LT *a, const LT *d, int V, int mode, floa
 template <typename LT, bool VECTOR, int K2_THREADS>
 __global__ void __launch_bounds__(K2_THREADS) epilogue_kernel(const VerifyParams p)
 {
-    const int b = blockIdx.x, tid = threadIdx.x;
+    // A cluster of CTAs per sequence (1 when the batch alone fills the GPU): they share the draw's walk over a row
+    // pair; everything else is evaluated alike by each of them and written by rank 0.
+    const int rank = (int)cluster_rank(), csize = (int)cluster_size();
+    const int b = (int)cluster_id(), tid = threadIdx.x;
     const int k = p.k, V = p.V, K = p.K;
     const float c = p.c;
     const LT *target = reinterpret_cast<const LT *>(p.target) + (size_t)b * (k + 1) * V;
@@ -521,7 +563,7 @@ __global__ void __launch_bounds__(K2_THREADS) epilogue_kernel(const VerifyParams
     __shared__ float sh_u;
     __shared__ uint32_t sh_flags;
     __shared__ double sh_reward;
-    __shared__ double sh_tot[K2_THREADS / 32];
+    __shared__ double sh_tot[64], sh_sub[K2_THREADS / 32];   // warp totals of the cluster / of the second level
     __shared__ int sh_accept[16];
     __shared__ double sh_align[16];
 
@@ -561,7 +603,7 @@ __global__ void __launch_bounds__(K2_THREADS) epilogue_kernel(const VerifyParams
         sh_accept[j] = accepted ? 1 : 0;
         sh_align[j] = align;
         if (flags) atomicOr(&sh_flags, flags);
-        if (p.diag) {
+        if (p.diag && rank == 0) {
             metasd_diag dg;
             dg.p_x = p_x; dg.q_x = q_x; dg.D = D; dg.u = u; dg.accept = accepted ? 1 : 0;
             p.diag[(size_t)b * k + j] = dg;
@@ -601,13 +643,16 @@ __global__ void __launch_bounds__(K2_THREADS) epilogue_kernel(const VerifyParams
         const LT *a = target + (size_t)n_acc * V;
         const LT *d = mode == 1 ? draft + (size_t)n_acc * V : nullptr;
         token = block_inverse_cdf<LT, VECTOR, K2_THREADS>(a, d, V, mode, sh_u, c, rs.max_a, rs.sum_a, rs.max_b, rs.sum_b,
-                                              sh_tot, &sh_tok);
+                                              sh_tot, sh_sub, &sh_tok, rank, csize);
         if (token < 0 && mode == 1)  // p == q in fp32 yet rejected: draw from p
             token = block_inverse_cdf<LT, VECTOR, K2_THREADS>(a, nullptr, V, 2, sh_u, c, rs.max_a, rs.sum_a, rs.max_b,
-                                                  rs.sum_b, sh_tot, &sh_tok);
+                                                  rs.sum_b, sh_tot, sh_sub, &sh_tok, rank, csize);
     }
 
-    if (tid == 0) {
+    // Rank 0 is about to advance the sequence's round counter and arm: every CTA of the cluster must have read
+    // the old ones first (they key its random numbers and pick its drafter), or the cluster would disagree.
+    cluster_sync_all();
+    if (tid == 0 && rank == 0) {
         const double r = sh_reward;
         p.accepted_len[b] = n_acc;
         p.next_token[b] = token;
@@ -628,7 +673,7 @@ __global__ void __launch_bounds__(K2_THREADS) epilogue_kernel(const VerifyParams
 template <typename LT>
 static cudaError_t launch_streaming_t(const VerifyParams &p, cudaStream_t stream, uint64_t *launches)
 {
-    dim3 g1(p.k + 1, p.batch), g2(p.batch);
+    dim3 g1(p.k + 1, p.batch);
     const bool big_ctas = p.batch <= 320;   // up to about two sequences per SM
     if (p.vector_ok && p.grp_size > 1) {
         const int n_items = p.batch * (p.k + 1);
@@ -647,11 +692,24 @@ static cudaError_t launch_streaming_t(const VerifyParams &p, cudaStream_t stream
     } else {
         row_stats_kernel<LT, false><<<g1, K1_THREADS, 0, stream>>>(p);
     }
-    if (p.vector_ok) {
-        if (big_ctas) epilogue_kernel<LT, true, 512><<<g2, 512, 0, stream>>>(p);
-        else epilogue_kernel<LT, true, 256><<<g2, 256, 0, stream>>>(p);
-    } else {
-        epilogue_kernel<LT, false, 256><<<g2, 256, 0, stream>>>(p);
+    {
+        // small batch: 4 CTAs of 512 threads per sequence; large batch: one CTA of 256 threads
+        const unsigned csize = big_ctas ? 4u : 1u, threads = big_ctas ? 512u : 256u;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)p.batch * csize);
+        cfg.blockDim = dim3(threads);
+        cfg.stream = stream;
+        cudaLaunchAttribute at;
+        at.id = cudaLaunchAttributeClusterDimension;
+        at.val.clusterDim.x = csize; at.val.clusterDim.y = 1; at.val.clusterDim.z = 1;
+        cfg.attrs = &at;
+        cfg.numAttrs = 1;
+        cudaError_t e;
+        if (!p.vector_ok) e = big_ctas ? cudaLaunchKernelEx(&cfg, epilogue_kernel<LT, false, 512>, p)
+                                       : cudaLaunchKernelEx(&cfg, epilogue_kernel<LT, false, 256>, p);
+        else e = big_ctas ? cudaLaunchKernelEx(&cfg, epilogue_kernel<LT, true, 512>, p)
+                          : cudaLaunchKernelEx(&cfg, epilogue_kernel<LT, true, 256>, p);
+        if (e != cudaSuccess) return e;
     }
     *launches += 2;
     return cudaGetLastError();
