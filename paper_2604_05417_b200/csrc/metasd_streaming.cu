@@ -382,24 +382,16 @@ __global__ void __launch_bounds__(KS_THREADS, 3) split_row_stats_kernel(const Ve
 // -------------------------------------------------------------------------------------------
 // K2
 // -------------------------------------------------------------------------------------------
-// weight of token v in the draw: mode 1 = max(0, p_v - q_v) (correction), mode 2 = p_v (bonus)
-template <typename LT, int VEC>
-__device__ __forceinline__ void draw_weights(const LT *a, const LT *d, int i, int mode, float c, float nma,
-                                             float ia, float nmb, float ib, float (&w)[VEC])
+// weight of token v in the draw: MODE 1 = max(0, p_v - q_v) (correction), MODE 2 = p_v (bonus)
+template <typename LT, int VEC, int MODE>
+__device__ __forceinline__ void weights_of(const float (&xa)[VEC], const float (&xb)[VEC], float c, float nma, float ia,
+                                           float nmb, float ib, float (&w)[VEC])
 {
-    float xa[VEC], xb[VEC];
-    if constexpr (VEC > 1) {
-        Logit<LT>::unpack(ld_stream(reinterpret_cast<const uint4 *>(a) + i), xa);
-        if (mode == 1) Logit<LT>::unpack(ld_stream(reinterpret_cast<const uint4 *>(d) + i), xb);
-    } else {
-        xa[0] = Logit<LT>::scalar(a, i);
-        if (mode == 1) xb[0] = Logit<LT>::scalar(d, i);
-    }
 #pragma unroll
     for (int e = 0; e < VEC; ++e) {
-        float pv = ex2(fmaf(xa[e], c, nma)) * ia;
-        if (mode == 1) {
-            float qv = ex2(fmaf(xb[e], c, nmb)) * ib;
+        const float pv = ex2(fmaf(xa[e], c, nma)) * ia;
+        if (MODE == 1) {
+            const float qv = ex2(fmaf(xb[e], c, nmb)) * ib;
             w[e] = fmaxf(pv - qv, 0.f);
         } else {
             w[e] = pv;
@@ -407,84 +399,160 @@ __device__ __forceinline__ void draw_weights(const LT *a, const LT *d, int i, in
     }
 }
 
+// one vector of logits as loaded (unpacked to fp32 only where it is used: registers)
+template <typename LT, int VEC> struct RawVec { uint4 v; };
+template <typename LT> struct RawVec<LT, 1> { float v; };
+
+template <typename LT, int VEC>
+__device__ __forceinline__ RawVec<LT, VEC> load_raw(const LT *row, int i)
+{
+    RawVec<LT, VEC> r;
+    if constexpr (VEC > 1) r.v = ld_stream(reinterpret_cast<const uint4 *>(row) + i);
+    else r.v = Logit<LT>::scalar(row, i);
+    return r;
+}
+
+template <typename LT, int VEC>
+__device__ __forceinline__ void unpack_raw(const RawVec<LT, VEC> &r, float (&x)[VEC])
+{
+    if constexpr (VEC > 1) Logit<LT>::unpack(r.v, x);
+    else x[0] = r.v;
+}
+
+template <typename LT, int VEC>
+__device__ __forceinline__ void draw_weights(const LT *a, const LT *d, int i, int mode, float c, float nma,
+                                             float ia, float nmb, float ib, float (&w)[VEC])
+{
+    float xa[VEC], xb[VEC];
+    unpack_raw<LT, VEC>(load_raw<LT, VEC>(a, i), xa);
+    if (mode == 1) {
+        unpack_raw<LT, VEC>(load_raw<LT, VEC>(d, i), xb);
+        weights_of<LT, VEC, 1>(xa, xb, c, nma, ia, nmb, ib, w);
+    } else {
+        weights_of<LT, VEC, 2>(xa, xa, c, nma, ia, nmb, ib, w);
+    }
+}
+
+// Sum of the draw's weights over the vectors [lo, hi), by one warp: lane l takes lo + l, lo + l + 32, ... and adds
+// each vector's fp32 sum to its fp64 total in that order.  Four vectors' loads are issued before the first is used.
+template <typename LT, int VEC, int MODE>
+__device__ __forceinline__ double warp_range_sum_m(const LT *a, const LT *d, int lo, int hi, float c, float nma,
+                                                   float ia, float nmb, float ib)
+{
+    constexpr int U = 4;
+    const int lane = threadIdx.x & 31;
+    double acc = 0.0;
+    for (int i0 = lo + lane; i0 < hi; i0 += 32 * U) {
+        RawVec<LT, VEC> ra[U], rb[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int i = i0 + 32 * u;
+            if (i < hi) {
+                ra[u] = load_raw<LT, VEC>(a, i);
+                if (MODE == 1) rb[u] = load_raw<LT, VEC>(d, i);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int i = i0 + 32 * u;
+            if (i < hi) {
+                float xa[VEC], xb[VEC], w[VEC];
+                unpack_raw<LT, VEC>(ra[u], xa);
+                if (MODE == 1) unpack_raw<LT, VEC>(rb[u], xb);
+                weights_of<LT, VEC, MODE>(xa, MODE == 1 ? xb : xa, c, nma, ia, nmb, ib, w);
+                float s = 0.f;
+#pragma unroll
+                for (int e = 0; e < VEC; ++e) s += w[e];
+                acc += (double)s;
+            }
+        }
+    }
+    return warp_sum(acc);
+}
+
+template <typename LT, int VEC>
+__device__ __forceinline__ double warp_range_sum(const LT *a, const LT *d, int lo, int hi, int mode, float c,
+                                                 float nma, float ia, float nmb, float ib)
+{
+    return mode == 1 ? warp_range_sum_m<LT, VEC, 1>(a, d, lo, hi, c, nma, ia, nmb, ib)
+                     : warp_range_sum_m<LT, VEC, 2>(a, d, lo, hi, c, nma, ia, nmb, ib);
+}
+
+// Given n <= 64 non-negative parts x[0..n) laid end to end after base0, finds the first part whose end lies beyond
+// the threshold; rounding may leave none, then the last part with mass (-1 if there is none).  FRACTION: the
+// threshold comes in as a fraction of the parts' sum and goes out absolute.  Returns the part, the sum of the parts
+// before it plus base0 in `base`, and the sum of all parts in `total`.  Every lane of the calling warp takes part
+// and gets the same answers.
+template <bool FRACTION>
+__device__ __forceinline__ int warp_find_part(const double *x, int n, double base0, double &threshold, double &base,
+                                              double &total)
+{
+    const unsigned FULL = 0xFFFFFFFFu;
+    const int lane = threadIdx.x & 31;
+    const double x0 = lane < n ? x[lane] : 0.0, x1 = lane + 32 < n ? x[lane + 32] : 0.0;
+    double i0 = x0, i1 = x1;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const double t0 = __shfl_up_sync(FULL, i0, o), t1 = __shfl_up_sync(FULL, i1, o);
+        if (lane >= o) { i0 += t0; i1 += t1; }
+    }
+    const double tot0 = __shfl_sync(FULL, i0, 31);
+    i1 += tot0;
+    total = __shfl_sync(FULL, i1, 31);
+    if (FRACTION) threshold *= total;
+    double e0 = __shfl_up_sync(FULL, i0, 1), e1 = __shfl_up_sync(FULL, i1, 1);
+    if (lane == 0) { e0 = 0.0; e1 = tot0; }
+    const unsigned c0 = __ballot_sync(FULL, lane < n && base0 + i0 > threshold);
+    const unsigned c1 = __ballot_sync(FULL, lane + 32 < n && base0 + i1 > threshold);
+    const unsigned m0 = __ballot_sync(FULL, x0 > 0.0), m1 = __ballot_sync(FULL, x1 > 0.0);
+    int part, src;
+    bool upper;
+    if (c0)      { src = __ffs(c0) - 1;    upper = false; }
+    else if (c1) { src = __ffs(c1) - 1;    upper = true; }
+    else if (m1) { src = 31 - __clz(m1);   upper = true; }
+    else if (m0) { src = 31 - __clz(m0);   upper = false; }
+    else { base = base0; return -1; }
+    part = src + (upper ? 32 : 0);
+    const double b0 = __shfl_sync(FULL, e0, src), b1 = __shfl_sync(FULL, e1, src);
+    base = base0 + (upper ? b1 : b0);
+    return part;
+}
+
 // Inverse CDF in token order over one row (pair): the smallest v with sum_{w<=v} weight_w > u * total.
 // Every warp owns a contiguous range of vectors; totals and offsets are carried in fp64.
 template <typename LT, bool VECTOR, int K2_THREADS>
 __device__ int block_inverse_cdf(const LT *a, const LT *d, int V, int mode, float u, float c, float max_a,
-                                 float sum_a, float max_b, float sum_b, double *sh_tot, double *sh_sub, int *sh_tok,
-                                 int rank, int csize)
+                                 float sum_a, float max_b, float sum_b, double *sh_tot, double *sh_sub, int *sh_tok)
 {
     constexpr int VEC = VECTOR ? Logit<LT>::VEC : 1;
     constexpr int NWARP = K2_THREADS / 32;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int nvec = V / VEC;
-    const int nwt = NWARP * csize, gw = rank * NWARP + warp;   // warps of the whole cluster, this warp among them
-    const int per_warp = (nvec + nwt - 1) / nwt;
-    const int v0 = min(gw * per_warp, nvec), v1 = min(v0 + per_warp, nvec);
+    const int per_warp = (nvec + NWARP - 1) / NWARP;
+    const int v0 = min(warp * per_warp, nvec), v1 = min(v0 + per_warp, nvec);
     const float nma = -max_a * c, nmb = -max_b * c;
     const float ia = 1.0f / sum_a, ib = 1.0f / sum_b;
 
-    double acc = 0.0;
-    for (int i = v0 + lane; i < v1; i += 32) {
-        float w[VEC];
-        draw_weights<LT, VEC>(a, d, i, mode, c, nma, ia, nmb, ib, w);
-        float s = 0.f;
-#pragma unroll
-        for (int e = 0; e < VEC; ++e) s += w[e];
-        acc += (double)s;
-    }
-    acc = warp_sum(acc);
-    // Every CTA of the cluster is running (a peer's shared memory may not be written before that) and has
-    // finished reading the slots of an earlier call.
-    cluster_sync_all();
-    // every CTA of the cluster gets every warp's total
-    if (lane < csize) st_cluster(map_to_rank(smem_addr(&sh_tot[gw]), (uint32_t)lane), acc);
+    const double acc = warp_range_sum<LT, VEC>(a, d, v0, v1, mode, c, nma, ia, nmb, ib);
+    if (lane == 0) sh_tot[warp] = acc;
     if (tid == 0) *sh_tok = -1;
-    cluster_sync_all();
-    double total = 0.0;
-    for (int w = 0; w < nwt; ++w) total += sh_tot[w];
-    if (!(total > 0.0)) { cluster_sync_all(); return -1; }
-    const double threshold = (double)u * total;
+    __syncthreads();
     // the warp whose range holds the crossing; rounding may leave none: then the last warp with mass
-    int wstar = -1, wlast = -1;
-    double base = 0.0, run = 0.0, base_last = 0.0;
-    for (int w = 0; w < nwt; ++w) {
-        if (sh_tot[w] > 0.0) { wlast = w; base_last = run; }
-        if (wstar < 0 && run + sh_tot[w] > threshold) { wstar = w; base = run; }
-        run += sh_tot[w];
-    }
-    if (wstar < 0) { wstar = wlast; base = base_last; }
-    // second level, in the CTA that owns that range: each of its warps takes a part of it, so that the final scan
-    // is a trip or two instead of a long chain of dependent loads in one warp
-    if (rank == wstar / NWARP) {
+    double threshold = (double)u, base, total;
+    const int wstar = warp_find_part<true>(sh_tot, NWARP, 0.0, threshold, base, total);
+    if (!(total > 0.0)) { __syncthreads(); return -1; }
+    // second level: each warp takes a part of that range, so that the final scan is a trip or two instead of a
+    // long chain of dependent loads in one warp
     const int r0 = min(wstar * per_warp, nvec), r1 = min(r0 + per_warp, nvec);
     const int per_sub = (r1 - r0 + NWARP - 1) / NWARP;
     const int s0 = min(r0 + warp * per_sub, r1), s1 = min(s0 + per_sub, r1);
     {
-        double acc2 = 0.0;
-        for (int i = s0 + lane; i < s1; i += 32) {
-            float w[VEC];
-            draw_weights<LT, VEC>(a, d, i, mode, c, nma, ia, nmb, ib, w);
-            float s = 0.f;
-#pragma unroll
-            for (int e = 0; e < VEC; ++e) s += w[e];
-            acc2 += (double)s;
-        }
-        acc2 = warp_sum(acc2);
+        const double acc2 = warp_range_sum<LT, VEC>(a, d, s0, s1, mode, c, nma, ia, nmb, ib);
         if (lane == 0) sh_sub[warp] = acc2;
     }
     __syncthreads();
-    int sstar = -1, slast = -1;
-    {
-        double run2 = base, base2 = base, base2_last = base;
-        for (int w = 0; w < NWARP; ++w) {
-            if (sh_sub[w] > 0.0) { slast = w; base2_last = run2; }
-            if (sstar < 0 && run2 + sh_sub[w] > threshold) { sstar = w; base2 = run2; }
-            run2 += sh_sub[w];
-        }
-        if (sstar < 0) { sstar = slast; base2 = base2_last; }
-        base = base2;
-    }
+    double total2;
+    const int sstar = warp_find_part<false>(sh_sub, NWARP, base, threshold, base, total2);
     if (warp == sstar) {
         const int v0 = s0, v1 = s1;
         int found = -1, last_pos = -1;
@@ -536,23 +604,18 @@ __device__ int block_inverse_cdf(const LT *a, const LT *d, int V, int mode, floa
             for (int o = 16; o > 0; o >>= 1) last_pos = max(last_pos, __shfl_xor_sync(0xFFFFFFFFu, last_pos, o));
             found = last_pos;
         }
-        // every CTA of the cluster gets the token: they must all agree on whether the draw found one
-        if (lane < csize) st_cluster(map_to_rank(smem_addr(sh_tok), (uint32_t)lane), (int32_t)found);
+        if (lane == 0) *sh_tok = found;
     }
-    }
-    cluster_sync_all();
+    __syncthreads();
     return *sh_tok;
 }
 
 // K2_THREADS: the draw walks one row pair per sequence, so a small batch wants large CTAs (many warps keep the
 // load chains short) and a large batch wants many small ones.
 template <typename LT, bool VECTOR, int K2_THREADS>
-__global__ void __launch_bounds__(K2_THREADS) epilogue_kernel(const VerifyParams p)
+__global__ void __launch_bounds__(K2_THREADS, 1024 / K2_THREADS) epilogue_kernel(const VerifyParams p)
 {
-    // A cluster of CTAs per sequence (1 when the batch alone fills the GPU): they share the draw's walk over a row
-    // pair; everything else is evaluated alike by each of them and written by rank 0.
-    const int rank = (int)cluster_rank(), csize = (int)cluster_size();
-    const int b = (int)cluster_id(), tid = threadIdx.x;
+    const int b = blockIdx.x, tid = threadIdx.x;
     const int k = p.k, V = p.V, K = p.K;
     const float c = p.c;
     const LT *target = reinterpret_cast<const LT *>(p.target) + (size_t)b * (k + 1) * V;
@@ -563,7 +626,7 @@ __global__ void __launch_bounds__(K2_THREADS) epilogue_kernel(const VerifyParams
     __shared__ float sh_u;
     __shared__ uint32_t sh_flags;
     __shared__ double sh_reward;
-    __shared__ double sh_tot[64], sh_sub[K2_THREADS / 32];   // warp totals of the cluster / of the second level
+    __shared__ double sh_tot[K2_THREADS / 32], sh_sub[K2_THREADS / 32];   // warp totals of the two search levels
     __shared__ int sh_accept[16];
     __shared__ double sh_align[16];
 
@@ -603,7 +666,7 @@ __global__ void __launch_bounds__(K2_THREADS) epilogue_kernel(const VerifyParams
         sh_accept[j] = accepted ? 1 : 0;
         sh_align[j] = align;
         if (flags) atomicOr(&sh_flags, flags);
-        if (p.diag && rank == 0) {
+        if (p.diag) {
             metasd_diag dg;
             dg.p_x = p_x; dg.q_x = q_x; dg.D = D; dg.u = u; dg.accept = accepted ? 1 : 0;
             p.diag[(size_t)b * k + j] = dg;
@@ -643,16 +706,15 @@ __global__ void __launch_bounds__(K2_THREADS) epilogue_kernel(const VerifyParams
         const LT *a = target + (size_t)n_acc * V;
         const LT *d = mode == 1 ? draft + (size_t)n_acc * V : nullptr;
         token = block_inverse_cdf<LT, VECTOR, K2_THREADS>(a, d, V, mode, sh_u, c, rs.max_a, rs.sum_a, rs.max_b, rs.sum_b,
-                                              sh_tot, sh_sub, &sh_tok, rank, csize);
-        if (token < 0 && mode == 1)  // p == q in fp32 yet rejected: draw from p
+                                              sh_tot, sh_sub, &sh_tok);
+        if (token < 0 && mode == 1) {  // p == q in fp32 yet rejected: draw from p
+            __syncthreads();   // every thread has read the first draw's answer before the slot is reused
             token = block_inverse_cdf<LT, VECTOR, K2_THREADS>(a, nullptr, V, 2, sh_u, c, rs.max_a, rs.sum_a, rs.max_b,
-                                                  rs.sum_b, sh_tot, sh_sub, &sh_tok, rank, csize);
+                                                  rs.sum_b, sh_tot, sh_sub, &sh_tok);
+        }
     }
 
-    // Rank 0 is about to advance the sequence's round counter and arm: every CTA of the cluster must have read
-    // the old ones first (they key its random numbers and pick its drafter), or the cluster would disagree.
-    cluster_sync_all();
-    if (tid == 0 && rank == 0) {
+    if (tid == 0) {
         const double r = sh_reward;
         p.accepted_len[b] = n_acc;
         p.next_token[b] = token;
@@ -693,23 +755,13 @@ static cudaError_t launch_streaming_t(const VerifyParams &p, cudaStream_t stream
         row_stats_kernel<LT, false><<<g1, K1_THREADS, 0, stream>>>(p);
     }
     {
-        // small batch: 4 CTAs of 512 threads per sequence; large batch: one CTA of 256 threads
-        const unsigned csize = big_ctas ? 4u : 1u, threads = big_ctas ? 512u : 256u;
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((unsigned)p.batch * csize);
-        cfg.blockDim = dim3(threads);
-        cfg.stream = stream;
-        cudaLaunchAttribute at;
-        at.id = cudaLaunchAttributeClusterDimension;
-        at.val.clusterDim.x = csize; at.val.clusterDim.y = 1; at.val.clusterDim.z = 1;
-        cfg.attrs = &at;
-        cfg.numAttrs = 1;
-        cudaError_t e;
-        if (!p.vector_ok) e = big_ctas ? cudaLaunchKernelEx(&cfg, epilogue_kernel<LT, false, 512>, p)
-                                       : cudaLaunchKernelEx(&cfg, epilogue_kernel<LT, false, 256>, p);
-        else e = big_ctas ? cudaLaunchKernelEx(&cfg, epilogue_kernel<LT, true, 512>, p)
-                          : cudaLaunchKernelEx(&cfg, epilogue_kernel<LT, true, 256>, p);
-        if (e != cudaSuccess) return e;
+        if (!p.vector_ok) {
+            if (big_ctas) epilogue_kernel<LT, false, 512><<<p.batch, 512, 0, stream>>>(p);
+            else epilogue_kernel<LT, false, 256><<<p.batch, 256, 0, stream>>>(p);
+        } else {
+            if (big_ctas) epilogue_kernel<LT, true, 512><<<p.batch, 512, 0, stream>>>(p);
+            else epilogue_kernel<LT, true, 256><<<p.batch, 256, 0, stream>>>(p);
+        }
     }
     *launches += 2;
     return cudaGetLastError();
