@@ -24,6 +24,7 @@ struct metasd_ctx {
     bool fused_ready;
     FusedPlan plan;
     int keep_permille;   // share of every row that the streaming kernel asks L2 to keep between its sweeps
+    int k1_stages;       // depth of the row-statistics kernel's cp.async pipeline (0 or 1: plain loads)
     // split streaming path
     int grp_size, grp_ctas;
     GroupRecord *grp_rec;
@@ -123,6 +124,10 @@ int metasd_init(metasd_ctx **out, const metasd_config *cfg)
         const char *kp = getenv("METASD_KEEP_PERMILLE");
         const int v = kp && *kp ? atoi(kp) : 650;
         c->keep_permille = v < 0 ? 0 : (v > 1000 ? 1000 : v);
+    }
+    {
+        const char *ks = getenv("METASD_K1_STAGES");
+        c->k1_stages = ks && *ks ? atoi(ks) : 0;
     }
     const size_t B = cfg->max_batch, K = cfg->n_drafters, tau = cfg->window, kp1 = cfg->max_draft + 1;
     cudaError_t e = cudaSuccess;
@@ -236,6 +241,7 @@ int metasd_verify(metasd_ctx *ctx, int32_t batch, int32_t k, const void *target_
     p.accepted_len = accepted_len; p.next_token = next_token; p.reward = reward; p.diag = diag;
     p.st = ctx->st; p.stats = ctx->stats; p.status = ctx->status;
     p.keep_permille = ctx->keep_permille;
+    p.k1_stages = ctx->k1_stages;
     p.grp_size = ctx->grp_size; p.grp_ctas = ctx->grp_ctas;
     p.grp_rec = ctx->grp_rec; p.grp_min = ctx->grp_min; p.grp_count = ctx->grp_count;
     const size_t row_bytes = (size_t)cfg.vocab * logit_size(cfg.logit_dtype);

@@ -162,6 +162,187 @@ __global__ void __launch_bounds__(K1_THREADS) row_stats_kernel(const VerifyParam
 }
 
 // -------------------------------------------------------------------------------------------
+// K1p
+// -------------------------------------------------------------------------------------------
+// K1 with its loads staged through shared memory.  Every thread copies its own vectors D - 1 trips ahead with
+// cp.async and reads them back when their group has landed; a slot is written and read by the same thread only, so
+// there is no barrier and no register cost.  The second sweep visits the thread's trips in reverse: the last D trips
+// of the first sweep are still in their slots and are not read from memory again, and each slot is refilled with the
+// trip D further down as soon as it has been used.  Vectors and their order per thread in sweep 1 are K1's; in
+// sweep 2 the partition of the row among threads differs from K1's, which only regroups an fp32 sum.
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, uint64_t policy)
+{
+    asm volatile("cp.async.cg.shared.global.L2::cache_hint [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "l"(policy) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ uint4 lds16(uint32_t addr)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+    return v;
+}
+
+template <typename LT, int D>
+__global__ void __launch_bounds__(K1_THREADS, 3) row_stats_staged_kernel(const VerifyParams p)
+{
+    static_assert((D & (D - 1)) == 0 && D >= 2, "stages: a power of two");
+    constexpr int VEC = Logit<LT>::VEC;
+    constexpr int NWARP = K1_THREADS / 32;
+    constexpr uint32_t ROW_STRIDE = K1_THREADS * 16, STAGE_STRIDE = 2 * ROW_STRIDE;
+    extern __shared__ __align__(16) unsigned char stage_mem[];   // [D][2 rows][K1_THREADS] 16-byte slots
+    const int j = blockIdx.x, b = blockIdx.y;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const float c = p.c;
+    const bool pair = j < p.k;
+
+    const uint4 *a4 = reinterpret_cast<const uint4 *>(reinterpret_cast<const LT *>(p.target) + ((size_t)b * (p.k + 1) + j) * p.V);
+    const uint4 *d4 = pair ? reinterpret_cast<const uint4 *>(draft_rows<LT>(p, b) + ((size_t)b * p.k + j) * p.V) : nullptr;
+    const int nvec = p.V / VEC;
+    const int n_trip = tid < nvec ? (nvec - tid + K1_THREADS - 1) / K1_THREADS : 0;   // vectors of this thread
+    const uint32_t slot0 = smem_addr(stage_mem) + (uint32_t)tid * 16u;
+
+    // ---- sweep 1: online (max, sum) of both rows, arg-max of the target row
+    MaxSum sa = {METASD_NEG_BIG, 0.f}, sb = {METASD_NEG_BIG, 0.f};
+    ArgMax am = {METASD_NEG_BIG, 0x7FFFFFFF};
+    const uint64_t keep = l2_policy_evict_last(), drop = l2_policy_evict_first();
+    const int keep_from = nvec - (int)((long long)nvec * p.keep_permille / 1000);
+    auto request1 = [&](int n) {   // one group per call, empty past the end: the group count stays in step
+        if (n < n_trip) {
+            const int i = tid + n * K1_THREADS;
+            const uint64_t pol = i >= keep_from ? keep : drop;
+            const uint32_t dst = slot0 + (uint32_t)(n & (D - 1)) * STAGE_STRIDE;
+            cp_async16(dst, a4 + i, pol);
+            if (pair) cp_async16(dst + ROW_STRIDE, d4 + i, pol);
+        }
+        cp_async_commit();
+    };
+#pragma unroll
+    for (int n = 0; n < D - 1; ++n) request1(n);
+    for (int n = 0; n < n_trip; ++n) {
+        request1(n + D - 1);
+        cp_async_wait<D - 1>();   // all but the D - 1 youngest groups have landed: trip n's is among them
+        const uint32_t src = slot0 + (uint32_t)(n & (D - 1)) * STAGE_STRIDE;
+        const int i = tid + n * K1_THREADS;
+        float xa[VEC];
+        Logit<LT>::unpack(lds16(src), xa);
+        float cm = xa[0];
+#pragma unroll
+        for (int e = 1; e < VEC; ++e) cm = fmaxf(cm, xa[e]);
+        if (cm > sa.m) {
+            sa.s *= ex2((sa.m - cm) * c);
+            sa.m = cm;
+            int first = 0;
+#pragma unroll
+            for (int e = VEC - 1; e >= 0; --e)
+                if (xa[e] == cm) first = e;
+            am.v = cm;
+            am.i = i * VEC + first;
+        }
+        const float nma = -sa.m * c;
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) sa.s += ex2(fmaf(xa[e], c, nma));
+        if (pair) {
+            float xb[VEC];
+            Logit<LT>::unpack(lds16(src + ROW_STRIDE), xb);
+            float bm = xb[0];
+#pragma unroll
+            for (int e = 1; e < VEC; ++e) bm = fmaxf(bm, xb[e]);
+            if (bm > sb.m) {
+                sb.s *= ex2((sb.m - bm) * c);
+                sb.m = bm;
+            }
+            const float nmb = -sb.m * c;
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) sb.s += ex2(fmaf(xb[e], c, nmb));
+        }
+    }
+    cp_async_wait<0>();
+
+    __shared__ MaxSum sh_a[NWARP], sh_b[NWARP];
+    __shared__ ArgMax sh_am[NWARP];
+    __shared__ double sh_min[NWARP];
+    __shared__ float sh_bcast[5];
+
+    sa = warp_merge(sa, c);
+    sb = warp_merge(sb, c);
+    am = warp_argmax(am);
+    if (lane == 0) { sh_a[warp] = sa; sh_b[warp] = sb; sh_am[warp] = am; }
+    __syncthreads();
+    if (warp == 0) {
+        MaxSum ra = lane < NWARP ? sh_a[lane] : MaxSum{METASD_NEG_BIG, 0.f};
+        MaxSum rb = lane < NWARP ? sh_b[lane] : MaxSum{METASD_NEG_BIG, 0.f};
+        ArgMax rm = lane < NWARP ? sh_am[lane] : ArgMax{METASD_NEG_BIG, 0x7FFFFFFF};
+        ra = warp_merge(ra, c);
+        rb = warp_merge(rb, c);
+        rm = warp_argmax(rm);
+        if (lane == 0) {
+            sh_bcast[0] = ra.m; sh_bcast[1] = ra.s; sh_bcast[2] = rb.m; sh_bcast[3] = rb.s;
+            sh_bcast[4] = -rb.m * c + log2f(ra.s / rb.s);
+            sh_am[0] = rm;
+        }
+    }
+    __syncthreads();
+    const float max_a = sh_bcast[0], sum_a = sh_bcast[1], max_b = sh_bcast[2], sum_b = sh_bcast[3];
+
+    // ---- sweep 2, this thread's trips in reverse: sum_v 2^min(ya_v, yb_v), one exponential per pair
+    double total_min = 0.0;
+    if (pair) {
+        const float nma = -max_a * c, nmb = sh_bcast[4];
+        const float ia = 1.0f / sum_a;
+        float acc = 0.f;
+        for (int n = n_trip - 1; n >= 0; --n) {
+            // the first D trips are still in their slots from sweep 1; the group of a later one was committed D trips
+            // ago, so at most D - 1 younger groups may still be pending
+            cp_async_wait<D - 1>();
+            const uint32_t src = slot0 + (uint32_t)(n & (D - 1)) * STAGE_STRIDE;
+            float xa[VEC], xb[VEC];
+            Logit<LT>::unpack(lds16(src), xa);
+            Logit<LT>::unpack(lds16(src + ROW_STRIDE), xb);
+#pragma unroll
+            for (int e = 0; e < VEC; ++e)
+                acc += ex2(fminf(fmaf(xa[e], c, nma), fmaf(xb[e], c, nmb)));
+            if (n >= D) {   // refill the slot just used with the trip D further down
+                const int i = tid + (n - D) * K1_THREADS;
+                cp_async16(src, a4 + i, drop);
+                cp_async16(src + ROW_STRIDE, d4 + i, drop);
+            }
+            cp_async_commit();
+        }
+        cp_async_wait<0>();
+        double w = warp_sum((double)(acc * ia));
+        if (lane == 0) sh_min[warp] = w;
+        __syncthreads();
+        if (tid == 0) {
+            for (int i = 0; i < NWARP; ++i) total_min += sh_min[i];
+        }
+    }
+
+    if (tid == 0) {
+        RowStats r;
+        r.max_a = max_a; r.sum_a = sum_a; r.max_b = max_b; r.sum_b = sum_b;
+        r.argmax_a = sh_am[0].i;
+        uint32_t flags = 0;
+        const bool bad_a = !(sum_a > 0.f) || !(sum_a < INFINITY) || !(max_a < INFINITY);
+        const bool bad_b = pair && (!(sum_b > 0.f) || !(sum_b < INFINITY) || !(max_b < INFINITY));
+        if (bad_a || bad_b) flags |= METASD_STATUS_NONFINITE;
+        r.sum_min = flags ? 0.0 : total_min;
+        r.flags = flags;
+        p.stats[(size_t)b * (p.k + 1) + j] = r;
+    }
+}
+
+template <typename LT, int D>
+static cudaError_t launch_staged(const VerifyParams &p, dim3 grid, cudaStream_t stream)
+{
+    const size_t smem = (size_t)D * 2 * K1_THREADS * 16;
+    cudaError_t e = cudaFuncSetAttribute(row_stats_staged_kernel<LT, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    row_stats_staged_kernel<LT, D><<<grid, K1_THREADS, smem, stream>>>(p);
+    return cudaSuccess;
+}
+
+// -------------------------------------------------------------------------------------------
 // K1s
 // -------------------------------------------------------------------------------------------
 constexpr int KS_THREADS = 512;
@@ -748,6 +929,9 @@ static cudaError_t launch_streaming_t(const VerifyParams &p, cudaStream_t stream
         void *args[] = {&q};
         e = cudaLaunchCooperativeKernel(reinterpret_cast<const void *>(&split_row_stats_kernel<LT>), dim3(n_groups * p.grp_size),
                                         dim3(KS_THREADS), args, 0, stream);
+        if (e != cudaSuccess) return e;
+    } else if (p.vector_ok && p.k1_stages > 1) {
+        cudaError_t e = p.k1_stages >= 4 ? launch_staged<LT, 4>(p, g1, stream) : launch_staged<LT, 2>(p, g1, stream);
         if (e != cudaSuccess) return e;
     } else if (p.vector_ok) {
         row_stats_kernel<LT, true><<<g1, K1_THREADS, 0, stream>>>(p);
