@@ -5,10 +5,10 @@
  * one speculative-decoding step -> block-divergence reward -> update the bandit") for a batch of
  * B independent sequences, each with its own bandit instance over K drafters:
  *
- *   metasd_select  : the drafter each sequence plays this round           (Algorithm 2, line 7)
- *   metasd_verify  : speculative-sampling verification of k drafted tokens (Algorithm 4, lines 6-12),
+ *   metasd_select  : the drafter each sequence plays this round           (Algorithm 2, selection rule)
+ *   metasd_verify  : speculative-sampling verification of k drafted tokens (Algorithm 4, verification loop),
  *                    the alignment reward (Definition 2, Eq. 4; or block efficiency, Sec. 2.3),
- *                    the bandit update (Algorithm 2, lines 9-10; Discounted UCB and Sliding-window
+ *                    the bandit update (Algorithm 2, statistics update; Discounted UCB and Sliding-window
  *                    UCB of the non-stationary appendix) and the next round's selection.
  *
  * Conventions
@@ -112,7 +112,7 @@ typedef struct metasd_diag {
 void metasd_default_config(metasd_config *cfg);
 
 /* Creates a context on cfg->device: validates cfg, allocates bandit state, scratch and (optionally)
- * staging, and resets every sequence (Algorithm 2, line 1: t <- 0).  *out is NULL on failure. */
+ * staging, and resets every sequence (Algorithm 2, initialisation: t <- 0).  *out is NULL on failure. */
 int metasd_init(metasd_ctx **out, const metasd_config *cfg);
 
 /* Frees everything metasd_init allocated.  NULL is accepted. */
@@ -123,14 +123,14 @@ void metasd_destroy(metasd_ctx *ctx);
  * or for all sequences when seq_ids is NULL.  Ids outside [0, max_batch) are ignored. */
 int metasd_reset(metasd_ctx *ctx, const int32_t *seq_ids, int32_t n, void *stream);
 
-/* Algorithm 2, lines 2-7: arm_out[b] = the drafter sequence b plays this round, b < batch.
+/* Algorithm 2, round-robin start and selection rule: arm_out[b] = the drafter sequence b plays this round, b < batch.
  * Rounds t < K play arm t (the initial sweep); afterwards argmax_i mu_i + beta sqrt(2 ln t / n_i),
  * lowest index on ties; an arm with no pull inside the SW-UCB window scores +infinity.  METASD_EXP3 and
  * METASD_RAND: the arm drawn as described at metasd_config. */
 int metasd_select(metasd_ctx *ctx, int32_t batch, int32_t *arm_out, void *stream);
 
-/* One verification round for sequences 0 .. batch-1 (Algorithm 4 lines 6-12, Definition 2,
- * Algorithm 2 lines 9-10, then the next selection).
+/* One verification round for sequences 0 .. batch-1 (Algorithm 4 verification loop, Definition 2,
+ * Algorithm 2 statistics update, then the next selection).
  *
  *   target_logits  [batch, k+1, V]  target logits at the k drafted positions and the bonus position
  *   draft_logits   [batch, k, V]    the played drafter's logits, already gathered by arm; or NULL and
@@ -187,7 +187,7 @@ uint64_t metasd_kernel_launches(const metasd_ctx *ctx);
 int metasd_resolved_path(const metasd_ctx *ctx, int32_t k);
 
 /* One verification round for callers that cannot allocate device memory.  (The paper has no
- * counterpart: this is a packaging of the stateless part of metasd_verify -- Algorithm 4 lines 6-12
+ * counterpart: this is a packaging of the stateless part of metasd_verify -- Algorithm 4's verification loop
  * and the reward -- for hosts where cudaMalloc is not available to this code: a serving process whose
  * memory pool already owns the whole device, a plugin that may not allocate after start-up, or a
  * latency-critical thread that must stay clear of the allocator.  Such callers cannot create a

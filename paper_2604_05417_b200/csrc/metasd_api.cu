@@ -122,12 +122,13 @@ int metasd_init(metasd_ctx **out, const metasd_config *cfg)
     c->cfg = *cfg;
     {   // 650: the best measured value on B200 for 128k-152k vocabularies (METASD_KEEP_PERMILLE overrides, for tuning)
         const char *kp = getenv("METASD_KEEP_PERMILLE");
-        const int v = kp && *kp ? atoi(kp) : 650;
+        const int v = kp && *kp ? atoi(kp) : (cfg->logit_dtype == METASD_BF16 ? 650 : 800);
         c->keep_permille = v < 0 ? 0 : (v > 1000 ? 1000 : v);
     }
     {
+        // 4: rows staged through shared memory; 0 (METASD_K1_STAGES=0, for comparison): plain loads
         const char *ks = getenv("METASD_K1_STAGES");
-        c->k1_stages = ks && *ks ? atoi(ks) : 0;
+        c->k1_stages = ks && *ks ? atoi(ks) : 4;
     }
     const size_t B = cfg->max_batch, K = cfg->n_drafters, tau = cfg->window, kp1 = cfg->max_draft + 1;
     cudaError_t e = cudaSuccess;

@@ -12,11 +12,11 @@
 //   - pass 2, over the same bytes still in shared memory, with the merged records of the whole row pair:
 //       sum_v min(p_v, q_v) = 1 - d_TV(p_j, q_j)  (Definition 2, Eq. 4), evaluated as
 //       sum_v 2^min(log2 p_v, log2 q_v): one exponential per PAIR;
-//     the accept test u q(x) < p(x) of the drafted token (Algorithm 4, lines 7-8), evaluated alike by
+//     the accept test u q(x) < p(x) of the drafted token (Algorithm 4, the accept step), evaluated alike by
 //     every thread of the cluster; at the first rejection (or the bonus position) the inverse-CDF draw
 //     from max(0, p - q) (or p), a prefix search in token order across the cluster (Algorithm 4, 11-12).
 // Rank 0 of the cluster then writes the outputs, forms the reward, and one warp updates the bandit and
-// selects the next arm with one lane per drafter (Algorithm 2, lines 7-10).
+// selects the next arm with one lane per drafter (Algorithm 2, update and selection steps).
 #include <limits.h>
 #include <stdio.h>
 #include <stdlib.h>
@@ -381,7 +381,7 @@ __device__ __forceinline__ Merged merge_records(const Exchange *rec, int n, int 
     return r;
 }
 
-// Bandit update and next selection by one warp, lane i = drafter i (Algorithm 2 lines 7-10; Discounted
+// Bandit update and next selection by one warp, lane i = drafter i (Algorithm 2, update and selection steps; Discounted
 // UCB; Sliding-window UCB).  Same fp64 expressions as the one-thread routines in metasd_device.cuh.
 __device__ void warp_bandit(const VerifyParams &p, int b, int t, int arm, double r)
 {
@@ -664,7 +664,7 @@ __global__ void __launch_bounds__(FUSED_MAX_THREADS, 2) fused_round_kernel(const
             rc.inv_sb = 1.0f / mg.Sb;
             rc.u_draw = sh.h_ud[j];
 
-            // ---- pass 2: sum_v min(p_v, q_v) of this warp's logits; the accept test of Algorithm 4 (lines 7-8),
+            // ---- pass 2: sum_v min(p_v, q_v) of this warp's logits; the accept test of Algorithm 4,
             //      evaluated alike by every thread of the cluster
             bool accepted = false;
             if (pair) {

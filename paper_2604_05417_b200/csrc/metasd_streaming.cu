@@ -1,17 +1,18 @@
 // Streaming path of the MetaSD verify round: works for every shape.
 //
-//   K1s split_row_stats_kernel  the same statistics as K1 with grp_size co-resident CTAs per row pair, each on its
-//                          own part of the vocabulary: they exchange (max, sum, arg-max) records through global
-//                          memory between the two sweeps.  Few enough row pairs are then in flight for the second
-//                          sweep to be served by L2 instead of HBM.  Used for 16-byte aligned rows when splitting pays.
 //   K1  row_stats_kernel   one CTA per (sequence b, position j): softmax statistics of the target
 //                          row and the draft row with an online maximum, the target arg-max, then
 //                          sum_v min(p_v, q_v) = 1 - d_TV(p_j, q_j) (Definition 2) in a second
-//                          sweep over the same rows.  Writes one RowStats record.
+//                          sweep over the same rows.  Writes one RowStats record.  Plain loads: any alignment.
+//   K1p row_stats_staged_kernel  K1 for 16-byte aligned rows (the default there): every thread stages its own
+//                          vectors through shared memory with cp.async, several trips ahead, and the second
+//                          sweep starts on the trips that are still staged instead of reading them again.
+//   K1s split_row_stats_kernel  (opt-in) K1 with grp_size co-resident CTAs per row pair, each on its own part
+//                          of the vocabulary, exchanging (max, sum, arg-max) records through global memory.
 //   K2  epilogue_kernel    one CTA per sequence: accept tests with the Philox uniforms (Algorithm 4,
-//                          lines 7-8), first rejection, inverse-CDF draw of the correction token from
-//                          max(0, p - q) or of the bonus token from p (lines 11-12), the reward, the
-//                          bandit update and the next round's arm (Algorithm 2, lines 7-10).
+//                          accept step), first rejection, inverse-CDF draw of the correction token from
+//                          max(0, p - q) or of the bonus token from p (its resampling step), the reward, the
+//                          bandit update and the next round's arm (Algorithm 2, update and selection steps).
 #include <stdlib.h>
 
 #include "metasd_device.cuh"
@@ -183,14 +184,14 @@ __device__ __forceinline__ uint4 lds16(uint32_t addr)
     return v;
 }
 
-template <typename LT, int D>
-__global__ void __launch_bounds__(K1_THREADS, 3) row_stats_staged_kernel(const VerifyParams p)
+template <typename LT, int D, int THREADS, int MINB>
+__global__ void __launch_bounds__(THREADS, MINB) row_stats_staged_kernel(const VerifyParams p)
 {
-    static_assert((D & (D - 1)) == 0 && D >= 2, "stages: a power of two");
+    static_assert(D >= 2, "at least two stages");
     constexpr int VEC = Logit<LT>::VEC;
-    constexpr int NWARP = K1_THREADS / 32;
-    constexpr uint32_t ROW_STRIDE = K1_THREADS * 16, STAGE_STRIDE = 2 * ROW_STRIDE;
-    extern __shared__ __align__(16) unsigned char stage_mem[];   // [D][2 rows][K1_THREADS] 16-byte slots
+    constexpr int NWARP = THREADS / 32;
+    constexpr uint32_t ROW_STRIDE = THREADS * 16, STAGE_STRIDE = 2 * ROW_STRIDE;
+    extern __shared__ __align__(16) unsigned char stage_mem[];   // [D][2 rows][THREADS] 16-byte slots
     const int j = blockIdx.x, b = blockIdx.y;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const float c = p.c;
@@ -199,7 +200,7 @@ __global__ void __launch_bounds__(K1_THREADS, 3) row_stats_staged_kernel(const V
     const uint4 *a4 = reinterpret_cast<const uint4 *>(reinterpret_cast<const LT *>(p.target) + ((size_t)b * (p.k + 1) + j) * p.V);
     const uint4 *d4 = pair ? reinterpret_cast<const uint4 *>(draft_rows<LT>(p, b) + ((size_t)b * p.k + j) * p.V) : nullptr;
     const int nvec = p.V / VEC;
-    const int n_trip = tid < nvec ? (nvec - tid + K1_THREADS - 1) / K1_THREADS : 0;   // vectors of this thread
+    const int n_trip = tid < nvec ? (nvec - tid + THREADS - 1) / THREADS : 0;   // vectors of this thread
     const uint32_t slot0 = smem_addr(stage_mem) + (uint32_t)tid * 16u;
 
     // ---- sweep 1: online (max, sum) of both rows, arg-max of the target row
@@ -209,9 +210,9 @@ __global__ void __launch_bounds__(K1_THREADS, 3) row_stats_staged_kernel(const V
     const int keep_from = nvec - (int)((long long)nvec * p.keep_permille / 1000);
     auto request1 = [&](int n) {   // one group per call, empty past the end: the group count stays in step
         if (n < n_trip) {
-            const int i = tid + n * K1_THREADS;
+            const int i = tid + n * THREADS;
             const uint64_t pol = i >= keep_from ? keep : drop;
-            const uint32_t dst = slot0 + (uint32_t)(n & (D - 1)) * STAGE_STRIDE;
+            const uint32_t dst = slot0 + (uint32_t)(n % D) * STAGE_STRIDE;
             cp_async16(dst, a4 + i, pol);
             if (pair) cp_async16(dst + ROW_STRIDE, d4 + i, pol);
         }
@@ -222,8 +223,8 @@ __global__ void __launch_bounds__(K1_THREADS, 3) row_stats_staged_kernel(const V
     for (int n = 0; n < n_trip; ++n) {
         request1(n + D - 1);
         cp_async_wait<D - 1>();   // all but the D - 1 youngest groups have landed: trip n's is among them
-        const uint32_t src = slot0 + (uint32_t)(n & (D - 1)) * STAGE_STRIDE;
-        const int i = tid + n * K1_THREADS;
+        const uint32_t src = slot0 + (uint32_t)(n % D) * STAGE_STRIDE;
+        const int i = tid + n * THREADS;
         float xa[VEC];
         Logit<LT>::unpack(lds16(src), xa);
         float cm = xa[0];
@@ -295,7 +296,7 @@ __global__ void __launch_bounds__(K1_THREADS, 3) row_stats_staged_kernel(const V
             // the first D trips are still in their slots from sweep 1; the group of a later one was committed D trips
             // ago, so at most D - 1 younger groups may still be pending
             cp_async_wait<D - 1>();
-            const uint32_t src = slot0 + (uint32_t)(n & (D - 1)) * STAGE_STRIDE;
+            const uint32_t src = slot0 + (uint32_t)(n % D) * STAGE_STRIDE;
             float xa[VEC], xb[VEC];
             Logit<LT>::unpack(lds16(src), xa);
             Logit<LT>::unpack(lds16(src + ROW_STRIDE), xb);
@@ -303,7 +304,7 @@ __global__ void __launch_bounds__(K1_THREADS, 3) row_stats_staged_kernel(const V
             for (int e = 0; e < VEC; ++e)
                 acc += ex2(fminf(fmaf(xa[e], c, nma), fmaf(xb[e], c, nmb)));
             if (n >= D) {   // refill the slot just used with the trip D further down
-                const int i = tid + (n - D) * K1_THREADS;
+                const int i = tid + (n - D) * THREADS;
                 cp_async16(src, a4 + i, drop);
                 cp_async16(src + ROW_STRIDE, d4 + i, drop);
             }
@@ -332,13 +333,13 @@ __global__ void __launch_bounds__(K1_THREADS, 3) row_stats_staged_kernel(const V
     }
 }
 
-template <typename LT, int D>
+template <typename LT, int D, int THREADS, int MINB>
 static cudaError_t launch_staged(const VerifyParams &p, dim3 grid, cudaStream_t stream)
 {
-    const size_t smem = (size_t)D * 2 * K1_THREADS * 16;
-    cudaError_t e = cudaFuncSetAttribute(row_stats_staged_kernel<LT, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    const size_t smem = (size_t)D * 2 * THREADS * 16;
+    cudaError_t e = cudaFuncSetAttribute(row_stats_staged_kernel<LT, D, THREADS, MINB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    row_stats_staged_kernel<LT, D><<<grid, K1_THREADS, smem, stream>>>(p);
+    row_stats_staged_kernel<LT, D, THREADS, MINB><<<grid, THREADS, smem, stream>>>(p);
     return cudaSuccess;
 }
 
@@ -816,7 +817,7 @@ __global__ void __launch_bounds__(K2_THREADS, 1024 / K2_THREADS) epilogue_kernel
     const int t = p.st.t[b];
     const int arm = p.st.arm[b];
     if (tid < k) {
-        // position j = tid: the accept test of Algorithm 4 (lines 7-8)
+        // position j = tid: the accept test of Algorithm 4
         const int j = tid;
         const int32_t *tokens = p.tokens + (p.token_arm_stride ? (size_t)arm * p.token_arm_stride : 0) + (size_t)b * k;
         const RowStats r = stats[j];
@@ -931,7 +932,12 @@ static cudaError_t launch_streaming_t(const VerifyParams &p, cudaStream_t stream
                                         dim3(KS_THREADS), args, 0, stream);
         if (e != cudaSuccess) return e;
     } else if (p.vector_ok && p.k1_stages > 1) {
-        cudaError_t e = p.k1_stages >= 4 ? launch_staged<LT, 4>(p, g1, stream) : launch_staged<LT, 2>(p, g1, stream);
+        // Measured on B200: bf16 rows (8 logits per 16 bytes) are bound by arithmetic as much as by memory and want
+        // many small CTAs (4 x 384 threads per SM); fp32 rows (4 logits per 16 bytes) are bound by memory and want
+        // few row pairs in flight and a large share of each kept in shared memory (1 x 1024 threads per SM).
+        cudaError_t e;
+        if (sizeof(LT) == 2) e = launch_staged<LT, 4, 384, 4>(p, g1, stream);
+        else e = launch_staged<LT, 4, 1024, 1>(p, g1, stream);
         if (e != cudaSuccess) return e;
     } else if (p.vector_ok) {
         row_stats_kernel<LT, true><<<g1, K1_THREADS, 0, stream>>>(p);
