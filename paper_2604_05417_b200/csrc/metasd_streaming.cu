@@ -936,7 +936,7 @@ static cudaError_t launch_streaming_t(const VerifyParams &p, cudaStream_t stream
         // many small CTAs (4 x 384 threads per SM); fp32 rows (4 logits per 16 bytes) are bound by memory and want
         // few row pairs in flight and a large share of each kept in shared memory (1 x 1024 threads per SM).
         cudaError_t e;
-        if (sizeof(LT) == 2) e = launch_staged<LT, 4, 384, 4>(p, g1, stream);
+        if constexpr (sizeof(LT) == 2) e = launch_staged<LT, 4, 384, 4>(p, g1, stream);
         else e = launch_staged<LT, 4, 1024, 1>(p, g1, stream);
         if (e != cudaSuccess) return e;
     } else if (p.vector_ok) {
