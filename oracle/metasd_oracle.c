@@ -34,6 +34,7 @@
 #define MSDO_SWUCB 2
 #define MSDO_EXP3 3
 #define MSDO_RAND 4
+#define MSDO_PETC 5
 /* position index of the random-number block that draws a randomised policy's arm */
 #define MSDO_SELECT_POSITION 0xFFFFFFFFu
 
@@ -296,6 +297,7 @@ void msdo_verify_sequence(const double *target, const double *draft, const int32
 /*       D-UCB: discounted reward sum S_i, discounted count N_i               */
 /*       EXP3 : weights w_i, kept divided by their largest (stat_b unused)    */
 /*       Rand : nothing                                                       */
+/*       PETC : this phase's reward sums R(i); membership of S (1 or 0)       */
 /*   win_arm[tau], win_reward[tau] (SW-UCB): round s sits in slot s mod tau   */
 /* ------------------------------------------------------------------------- */
 
@@ -378,11 +380,93 @@ int msdo_random_select(int variant, int K, double gamma, int t, const double *st
     return arm;
 }
 
+/* ---- Pure exploration-then-commit (algorithm "Pure exploration-then-commit (PETC)") with Sequential
+ * Halving (algorithm "Sequential Halving (SH)") as its exploration phase.
+ * One SH run with a total budget of T = `budget` rounds, then the surviving drafter for every later round.
+ * SH: S_0 = [K]; in phase r every drafter of S_r is pulled n_r = floor(T / (|S_r| L)) more times and
+ * R_r(i) sums the rewards of those pulls only; S_{r+1} keeps the ceil(|S_r| / 2) drafters of S_r with the
+ * largest R_r.  Readings (the printed box is garbled in three places): L = ceil(log2 K) phases, as in the
+ * cited algorithm, so that exactly one drafter survives for every K (the box prints floor); the half that is
+ * kept is the one with the LARGER sums (the box's inequality would keep the worse half); n_r is at least 1.
+ * Within a phase the members of S_r are pulled in index order, n_r consecutive rounds each (fewest switches);
+ * equal sums: the lower index is kept. */
+int msdo_sh_phases(int K)
+{
+    int L = 0, size = K;
+    while (size > 1) { size = (size + 1) / 2; ++L; }
+    return L;
+}
+
+int msdo_sh_pulls(int budget, int size, int L)
+{
+    int n = budget / (size * L);
+    return n < 1 ? 1 : n;
+}
+
+/* Where round t falls: *phase = r, or L once exploration is over; for r < L also the first round of the phase,
+ * |S_r| and n_r. */
+void msdo_sh_locate(int K, int budget, int t, int *phase, int *first, int *size, int *pulls)
+{
+    const int L = msdo_sh_phases(K);
+    int start = 0, members = K;
+    for (int r = 0; r < L; ++r) {
+        const int n = msdo_sh_pulls(budget, members, L);
+        if (t < start + n * members) { *phase = r; *first = start; *size = members; *pulls = n; return; }
+        start += n * members;
+        members = (members + 1) / 2;
+    }
+    *phase = L; *first = start; *size = members; *pulls = 0;
+}
+
+/* The drafter of round t: during phase r the ((t - first) / n_r)-th member of S_r in index order; afterwards
+ * the survivor. */
+int msdo_petc_select(int K, int budget, int t, const double *member)
+{
+    int phase, first, size, pulls, which = 0;
+    msdo_sh_locate(K, budget, t, &phase, &first, &size, &pulls);
+    if (phase < msdo_sh_phases(K)) which = (t - first) / pulls;
+    for (int i = 0; i < K; ++i) {
+        if (member[i] > 0.0) {
+            if (which == 0) return i;
+            --which;
+        }
+    }
+    return K - 1;   /* not reached while S is consistent with t */
+}
+
+/* Adds the reward of round t (arm a) to R; if that round closed a phase, halves S and clears R.
+ * margin (optional): smallest kept sum minus largest dropped sum of that halving, else +infinity. */
+void msdo_petc_update(int K, int budget, int t, double *R, double *member, int a, double r, double *margin)
+{
+    int phase, first, size, pulls;
+    if (margin) *margin = INFINITY;
+    R[a] += r;
+    msdo_sh_locate(K, budget, t, &phase, &first, &size, &pulls);
+    if (phase >= msdo_sh_phases(K) || t + 1 != first + size * pulls) return;
+    const int keep = (size + 1) / 2;
+    double kept[64], worst_kept = INFINITY, best_dropped = -INFINITY;
+    for (int i = 0; i < K; ++i) kept[i] = 0.0;
+    for (int c = 0; c < keep; ++c) {              /* the largest remaining sum, lowest index first */
+        int best = -1;
+        for (int i = 0; i < K; ++i)
+            if (member[i] > 0.0 && kept[i] == 0.0 && (best < 0 || R[i] > R[best])) best = i;
+        kept[best] = 1.0;
+        if (R[best] < worst_kept) worst_kept = R[best];
+    }
+    for (int i = 0; i < K; ++i)
+        if (member[i] > 0.0 && kept[i] == 0.0 && R[i] > best_dropped) best_dropped = R[i];
+    if (margin && size > keep) *margin = worst_kept - best_dropped;
+    for (int i = 0; i < K; ++i) { member[i] = kept[i]; R[i] = 0.0; }
+}
+
 /* The update after a round with arm a and reward r. */
 void msdo_bandit_update(int variant, int K, double gamma, int tau, int32_t *t, double *stat_a,
-                        double *stat_b, int32_t *win_arm, double *win_reward, int a, double r)
+                        double *stat_b, int32_t *win_arm, double *win_reward, int a, double r, double *margin)
 {
-    if (variant == MSDO_UCB) {
+    if (margin) *margin = INFINITY;
+    if (variant == MSDO_PETC) {
+        msdo_petc_update(K, tau, *t, stat_a, stat_b, a, r, margin);    /* tau carries the exploration budget */
+    } else if (variant == MSDO_UCB) {
         /* mu_hat <- (mu_hat * n + r) / (n + 1); n <- n + 1 */
         stat_a[a] = (stat_a[a] * stat_b[a] + r) / (stat_b[a] + 1.0);
         stat_b[a] = stat_b[a] + 1.0;
@@ -455,7 +539,10 @@ void msdo_select_batch(int B, int variant, int K, double beta, double gamma, int
                        const int32_t *win_arm, const double *win_reward, int32_t *arm, double *gap)
 {
     for (int b = 0; b < B; ++b) {
-        if (variant == MSDO_EXP3 || variant == MSDO_RAND)
+        if (variant == MSDO_PETC) {
+            arm[b] = msdo_petc_select(K, tau, t[b], stat_b + (size_t)b * K);
+            if (gap) gap[b] = INFINITY;
+        } else if (variant == MSDO_EXP3 || variant == MSDO_RAND)
             arm[b] = msdo_random_select(variant, K, gamma, t[b], stat_a + (size_t)b * K, seed,
                                         sequence_base + (uint32_t)b, gap ? gap + b : NULL);
         else
@@ -467,12 +554,13 @@ void msdo_select_batch(int B, int variant, int K, double beta, double gamma, int
 
 void msdo_update_batch(int B, int variant, int K, double gamma, int tau, int32_t *t, double *stat_a,
                        double *stat_b, int32_t *win_arm, double *win_reward, const int32_t *arm,
-                       const double *reward)
+                       const double *reward, double *margin)
 {
     for (int b = 0; b < B; ++b)
         msdo_bandit_update(variant, K, gamma, tau, t + b, stat_a + (size_t)b * K, stat_b + (size_t)b * K,
                            win_arm ? win_arm + (size_t)b * tau : NULL,
-                           win_reward ? win_reward + (size_t)b * tau : NULL, arm[b], reward[b]);
+                           win_reward ? win_reward + (size_t)b * tau : NULL, arm[b], reward[b],
+                           margin ? margin + b : NULL);
 }
 
 int msdo_max_threads(void)

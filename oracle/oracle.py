@@ -21,7 +21,7 @@ _SRC = os.path.join(_HERE, "metasd_oracle.c")
 _LIB = os.path.join(_HERE, "libmetasd_oracle.so")
 
 DTYPE_BF16, DTYPE_FP32 = 0, 1
-UCB, DUCB, SWUCB, EXP3, RAND = 0, 1, 2, 3, 4
+UCB, DUCB, SWUCB, EXP3, RAND, PETC = 0, 1, 2, 3, 4, 5
 REWARD_BD, REWARD_BE = 0, 1
 STATUS_NONFINITE, STATUS_TOKEN_OOR, STATUS_Q_ZERO = 1, 2, 4
 
@@ -172,7 +172,7 @@ class OracleConfig:
     bandit: int = UCB
     beta: float = 0.01
     gamma: float = 0.975      # D-UCB discount
-    tau: int = 50             # SW-UCB window
+    tau: int = 50             # SW-UCB window; PETC: the exploration budget in rounds
     reward: int = REWARD_BD
     reward_temperature: float = 1.0
     sequence_base: int = 0
@@ -194,12 +194,16 @@ class OracleMetaSD:
         self.select_seed = 0            # key of a randomised policy's arm draw: 0 until the first verify call,
         if cfg.bandit == EXP3:          # then the seed of the latest one
             self.stat_a[:] = 1.0
+        if cfg.bandit == PETC:          # S_0 = [K]
+            self.stat_b[:] = 1.0
+        self.halving_margin = np.full(B, np.inf)    # PETC: the closest call of any halving so far
 
     def reset(self, seq_ids=None):
         ids = slice(None) if seq_ids is None else np.asarray(seq_ids)
         self.t[ids] = 0
         self.stat_a[ids] = 1.0 if self.cfg.bandit == EXP3 else 0.0      # EXP3: w_0(i) = 1
-        self.stat_b[ids] = 0
+        self.stat_b[ids] = 1.0 if self.cfg.bandit == PETC else 0.0     # PETC: every drafter is in S_0
+        self.halving_margin[ids] = np.inf
         self.win_arm[ids] = 0
         self.win_reward[ids] = 0
 
@@ -213,7 +217,7 @@ class OracleMetaSD:
                                 C.c_uint64(self.select_seed), C.c_uint32(c.sequence_base), _p(self.t),
                                 _p(self.stat_a), _p(self.stat_b), _p(self.win_arm),
                                 _p(self.win_reward), _p(arm), _p(gap))
-        self.last_gap[:B] = gap
+        self.last_gap[:B] = np.minimum(gap, self.halving_margin[:B]) if c.bandit == PETC else gap
         return arm
 
     def verify(self, target_logits, draft_logits, draft_tokens, temperature, seed,
@@ -267,10 +271,12 @@ class OracleMetaSD:
         B = len(arm)
         arm = np.ascontiguousarray(arm, dtype=np.int32)
         reward = _f64(reward)
+        margin = np.full(B, np.inf)
         lib().msdo_update_batch(C.c_int(B), C.c_int(c.bandit), C.c_int(c.n_drafters),
                                 C.c_double(c.gamma), C.c_int(max(c.tau, 1)), _p(self.t),
                                 _p(self.stat_a), _p(self.stat_b), _p(self.win_arm),
-                                _p(self.win_reward), _p(arm), _p(reward))
+                                _p(self.win_reward), _p(arm), _p(reward), _p(margin))
+        self.halving_margin[:B] = np.minimum(self.halving_margin[:B], margin)
 
     def mean_estimates(self):
         """mu_hat and n per arm, as the selection rule sees them (for tests)."""

@@ -220,6 +220,7 @@ __global__ void __launch_bounds__(THREADS, MINB) row_stats_staged_kernel(const V
     };
 #pragma unroll
     for (int n = 0; n < D - 1; ++n) request1(n);
+#pragma unroll 4
     for (int n = 0; n < n_trip; ++n) {
         request1(n + D - 1);
         cp_async_wait<D - 1>();   // all but the D - 1 youngest groups have landed: trip n's is among them
@@ -292,6 +293,7 @@ __global__ void __launch_bounds__(THREADS, MINB) row_stats_staged_kernel(const V
         const float nma = -max_a * c, nmb = sh_bcast[4];
         const float ia = 1.0f / sum_a;
         float acc = 0.f;
+#pragma unroll 4
         for (int n = n_trip - 1; n >= 0; --n) {
             // the first D trips are still in their slots from sweep 1; the group of a later one was committed D trips
             // ago, so at most D - 1 younger groups may still be pending

@@ -1,4 +1,4 @@
-"""Pins of the CPU oracle's bandit policies (MetaSD-UCB, Discounted UCB, Sliding-window UCB).
+"""Pins of the CPU oracle's bandit policies (MetaSD-UCB, Discounted UCB, Sliding-window UCB, EXP3, Rand, PETC).
 
 Expected values are invariants, textbook consequences of the index rule, the explicit-constant
 pull bound the paper quotes, and reductions between the variants -- never the oracle's own output.
@@ -313,3 +313,78 @@ def test_rand_is_floor_of_u_times_k_in_integers_and_uniform():
     before = o.stat_a.copy()
     o.update(arm, np.ones(B))
     assert np.array_equal(o.stat_a, before) and (o.t == np.arange(B) % 17 + 1).all()   # no statistics, t advances
+
+
+# ---------------------------------------------------------------------------------------------
+# Pure exploration-then-commit with Sequential Halving (the two algorithm boxes of the switching-cost appendix)
+# ---------------------------------------------------------------------------------------------
+def test_petc_schedule_worked_by_hand_for_four_drafters():
+    # K = 4, budget 16: L = 2 phases; phase 0: floor(16 / (4 * 2)) = 2 pulls each of 0,1,2,3;
+    # phase 1: floor(16 / (2 * 2)) = 4 pulls each of the two with the larger phase-0 sums; then the winner.
+    means = [0.2, 0.9, 0.4, 0.7]
+    arms, _, _ = run_bandit(O.PETC, 4, lambda a, t, g: means[a], 30, tau=16)
+    assert arms[:8].tolist() == [0, 0, 1, 1, 2, 2, 3, 3]
+    assert arms[8:16].tolist() == [1, 1, 1, 1, 3, 3, 3, 3]          # survivors in index order
+    assert (arms[16:] == 1).all()                                     # committed to the best
+
+
+def test_petc_phase_sums_restart_and_only_the_current_phase_counts():
+    # drafter 3 is best in phase 0 and worst afterwards: with sums restarted it loses phase 1 to drafter 1
+    def reward(a, t, g):
+        if a == 3:
+            return 1.0 if t < 8 else 0.0
+        return [0.1, 0.6, 0.2][a]
+    arms, _, orc = run_bandit(O.PETC, 4, reward, 20, tau=16)
+    assert sorted(set(arms[8:16].tolist())) == [1, 3]
+    assert (arms[16:] == 1).all()
+    assert orc.stat_b[0].tolist() == [0.0, 1.0, 0.0, 0.0]             # S after the last halving
+
+
+@pytest.mark.parametrize("K", [1, 2, 3, 5, 6, 7, 8, 9, 16])
+def test_petc_halves_ceil_log2_times_and_spends_at_most_its_budget(K):
+    budget = 12 * K
+    L = math.ceil(math.log2(K)) if K > 1 else 0
+    rng_means = np.random.RandomState(K).rand(K)
+    arms, _, orc = run_bandit(O.PETC, K, lambda a, t, g: rng_means[a] + 0.01 * g.rand(), budget + 25, tau=budget)
+    # exploration length: sum over phases of n_r |S_r| with |S_{r+1}| = ceil(|S_r| / 2)
+    size, spent, sizes = K, 0, []
+    for _ in range(L):
+        sizes.append(size)
+        spent += (budget // (size * L)) * size
+        size = (size + 1) // 2
+    assert size == 1 and spent <= budget
+    tail = arms[spent:]
+    assert (tail == tail[0]).all()                                    # one drafter for every later round
+    assert int(orc.stat_b[0].sum()) == 1 and orc.stat_b[0][tail[0]] == 1.0
+    # inside phase r exactly |S_r| distinct drafters are played, each the same number of times
+    pos = 0
+    for s in sizes:
+        n = budget // (s * L)
+        block = arms[pos:pos + n * s]
+        values, counts = np.unique(block, return_counts=True)
+        assert len(values) == s and (counts == n).all()
+        pos += n * s
+    # with well separated means the best drafter survives
+    assert tail[0] == int(np.argmax(rng_means))
+
+
+def test_petc_keeps_the_lower_index_on_equal_sums_and_pulls_at_least_once():
+    arms, _, orc = run_bandit(O.PETC, 4, lambda a, t, g: 0.5, 12, tau=1)     # budget too small: n_r = 1
+    assert arms[:4].tolist() == [0, 1, 2, 3] and arms[4:6].tolist() == [0, 1]
+    assert (arms[6:] == 0).all()
+
+
+def test_sequential_halving_error_rate_respects_the_bound_the_paper_quotes():
+    # P(wrong survivor) <= 3 log2(K) exp(-T / (8 H2 log2 K)), H2 = max_i i / Delta_i^2 (gaps sorted increasingly)
+    means = np.array([0.9, 0.5, 0.45, 0.4])
+    K, T = 4, 1600
+    gaps = np.sort(means.max() - means)[1:]                                  # Delta_(2) <= ... <= Delta_(K)
+    H2 = max((i + 2) / gaps[i] ** 2 for i in range(K - 1))
+    bound = 3 * math.log2(K) * math.exp(-T / (8 * H2 * math.log2(K)))
+    assert bound < 0.02                                                      # not a vacuous statement
+    wrong, runs = 0, 150
+    for s in range(runs):
+        arms, _, _ = run_bandit(O.PETC, K, lambda a, t, g: float(g.rand() < means[a]), T + 1, tau=T, seed=s)
+        wrong += int(arms[-1] != 0)
+    assert wrong / runs <= bound + 3 * math.sqrt(max(bound * (1 - bound), 1e-4) / runs)
+    assert wrong / runs < 0.05                                               # and it does find the best drafter
