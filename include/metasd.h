@@ -53,7 +53,12 @@ enum metasd_bandit {
     METASD_SWUCB = 2, /* Sliding-window UCB (non-stationary appendix) */
     METASD_EXP3 = 3,  /* MetaSD-EXP3 (the algorithm box of that name): arms drawn from
                          p_t(i) = (1 - gamma) w_i / sum w + gamma / K, w_a <- w_a exp(gamma (r / p_t(a)) / K) */
-    METASD_RAND = 4   /* the uniformly random baseline of the paper's tables */
+    METASD_RAND = 4,  /* the uniformly random baseline of the paper's tables */
+    METASD_PETC = 5   /* Pure exploration-then-commit (the algorithm box of that name): one Sequential Halving run
+                         (the box of that name) over `window` rounds, then the surviving drafter only.
+                         ceil(log2 K) phases; every surviving drafter is played floor(window / (survivors * phases))
+                         times per phase (at least once), in index order, one block of rounds each; the half with the
+                         larger phase sums survives, the lower index on equal sums */
 };
 enum metasd_reward { METASD_REWARD_BD = 0, METASD_REWARD_BE = 1 };
 
@@ -76,7 +81,8 @@ enum metasd_path {
 
 /* Hyper-parameters of metasd_init.  Paper notation: n_drafters = K, max_draft = N_max, beta = the
  * exploration strength of Algorithm 2 (experiments: 0.01), gamma = the D-UCB decay or, for METASD_EXP3, its
- * mixing parameter (both are called gamma in the paper), window = the SW-UCB window tau (none of these values
+ * mixing parameter (both are called gamma in the paper), window = the SW-UCB window tau or, for METASD_PETC, its
+ * exploration budget in rounds (none of these values
  * is given in the paper; 0.975 / 50 are this library's defaults).
  * The randomised policies draw the arm of round t from word 2 of the Philox block keyed by the seed of the
  * latest metasd_verify call (0 before the first one) at counter (sequence_base + b, t, 0xFFFFFFFF, 0):
@@ -89,7 +95,7 @@ typedef struct metasd_config {
     int32_t logit_dtype;        /* metasd_dtype */
     int32_t bandit;             /* metasd_bandit */
     int32_t reward;             /* metasd_reward */
-    int32_t window;             /* tau >= 1 (used by METASD_SWUCB) */
+    int32_t window;             /* tau >= 1 (METASD_SWUCB), exploration rounds (METASD_PETC) */
     int32_t device;             /* CUDA device ordinal */
     int32_t path;               /* metasd_path */
     uint32_t sequence_base;     /* id of sequence 0 in the random-number key (batch sharding) */

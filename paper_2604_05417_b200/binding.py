@@ -17,14 +17,14 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libmetasd.so")
 
 BF16, FP32 = 0, 1
-UCB, DUCB, SWUCB, EXP3, RAND = 0, 1, 2, 3, 4
+UCB, DUCB, SWUCB, EXP3, RAND, PETC = 0, 1, 2, 3, 4, 5
 REWARD_BD, REWARD_BE = 0, 1
 PATH_AUTO, PATH_STREAMING, PATH_FUSED = 0, 1, 2
 STATUS_NONFINITE, STATUS_TOKEN_OOR, STATUS_Q_ZERO, STATUS_TIMEOUT, STATUS_BAD_POINTER = 1, 2, 4, 8, 16
 
 OK, ERR_INVALID_ARGUMENT, ERR_UNSUPPORTED, ERR_CUDA, ERR_NO_MEMORY, ERR_BAD_STATE_BLOB = 0, -1, -2, -3, -4, -5
 
-BANDITS = {"ucb": UCB, "ducb": DUCB, "swucb": SWUCB, "exp3": EXP3, "rand": RAND}
+BANDITS = {"ucb": UCB, "ducb": DUCB, "swucb": SWUCB, "exp3": EXP3, "rand": RAND, "petc": PETC}
 DTYPES = {"bf16": BF16, "fp32": FP32, torch.bfloat16: BF16, torch.float32: FP32}
 
 EXPORTS = (

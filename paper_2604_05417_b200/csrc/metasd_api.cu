@@ -58,7 +58,7 @@ int validate_config(const metasd_config *c)
     if (c->max_draft < 1 || c->max_draft > 16) return METASD_ERR_INVALID_ARGUMENT;
     if (c->vocab < 1) return METASD_ERR_INVALID_ARGUMENT;
     if (c->logit_dtype != METASD_BF16 && c->logit_dtype != METASD_FP32) return METASD_ERR_UNSUPPORTED;
-    if (c->bandit < METASD_UCB || c->bandit > METASD_RAND) return METASD_ERR_UNSUPPORTED;
+    if (c->bandit < METASD_UCB || c->bandit > METASD_PETC) return METASD_ERR_UNSUPPORTED;
     if (c->reward != METASD_REWARD_BD && c->reward != METASD_REWARD_BE) return METASD_ERR_UNSUPPORTED;
     if (c->path < METASD_PATH_AUTO || c->path > METASD_PATH_FUSED) return METASD_ERR_UNSUPPORTED;
     if (c->window < 1 || c->window > (1 << 20)) return METASD_ERR_INVALID_ARGUMENT;

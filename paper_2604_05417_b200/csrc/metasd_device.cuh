@@ -300,12 +300,63 @@ __device__ inline int random_select(int variant, int K, double gamma, int t, con
     return K - 1;
 }
 
+// Pure exploration-then-commit with Sequential Halving (the algorithm boxes of those names): one halving run over
+// `budget` rounds, then the surviving drafter.  ceil(log2 K) phases; in a phase every member of the surviving set
+// is played floor(budget / (members * phases)) times (at least once), members in index order, each in one block.
+// sa: the current phase's reward sums; sb: membership of the surviving set (1 or 0).
+struct HalvingPhase {
+    int index, n_phases, first, members, pulls;   // index == n_phases: exploration is over
+};
+__device__ inline HalvingPhase halving_phase(int K, int budget, int t)
+{
+    HalvingPhase ph;
+    ph.n_phases = K > 1 ? 32 - __clz(K - 1) : 0;
+    ph.first = 0;
+    ph.members = K;
+    for (ph.index = 0; ph.index < ph.n_phases; ++ph.index) {
+        ph.pulls = max(budget / (ph.members * ph.n_phases), 1);
+        const int length = ph.pulls * ph.members;
+        if (t - ph.first < length) return ph;
+        ph.first += length;
+        ph.members = (ph.members + 1) >> 1;
+    }
+    ph.pulls = 0;
+    return ph;
+}
+__device__ inline int petc_select(int K, int budget, int t, const double *sb)
+{
+    const HalvingPhase ph = halving_phase(K, budget, t);
+    int skip = ph.index < ph.n_phases ? (t - ph.first) / ph.pulls : 0;
+    for (int i = 0; i < K; ++i)
+        if (sb[i] > 0.0 && skip-- == 0) return i;
+    return K - 1;
+}
+__device__ inline void petc_update(int K, int budget, int t, double *sa, double *sb, int a, double r)
+{
+    sa[a] += r;
+    const HalvingPhase ph = halving_phase(K, budget, t);
+    if (ph.index >= ph.n_phases || t + 1 != ph.first + ph.pulls * ph.members) return;
+    // the round closed a phase: the better half stays (larger sum; the lower index on equal sums)
+    uint32_t in = 0, out = 0;
+    for (int i = 0; i < K; ++i)
+        if (sb[i] > 0.0) in |= 1u << i;
+    for (int c = (ph.members + 1) >> 1; c > 0; --c) {
+        int best = -1;
+        for (int i = 0; i < K; ++i)
+            if (((in >> i) & 1u) && (best < 0 || sa[i] > sa[best])) best = i;
+        in &= ~(1u << best);
+        out |= 1u << best;
+    }
+    for (int i = 0; i < K; ++i) { sb[i] = (out >> i) & 1u ? 1.0 : 0.0; sa[i] = 0.0; }
+}
+
 // Arm for round t of one sequence.  sa/sb: this sequence's [K] statistics; wa/wr: its window.
 __device__ inline int bandit_select(int variant, int K, double beta, double gamma, int tau, int t, const double *sa,
                                     const double *sb, const int32_t *wa, const double *wr, uint64_t seed,
                                     uint32_t sequence)
 {
     if (variant == METASD_EXP3 || variant == METASD_RAND) return random_select(variant, K, gamma, t, sa, seed, sequence);
+    if (variant == METASD_PETC) return petc_select(K, tau, t, sb);   // tau carries the exploration budget
     if (t < K) return t;  // initial sweep: every drafter once, in order
     double mu[16], n[16];
     if (variant == METASD_SWUCB) {
@@ -356,6 +407,8 @@ __device__ inline void bandit_update(int variant, int K, double gamma, int tau, 
         for (int i = 0; i < K; ++i) sa[i] /= top;
     } else if (variant == METASD_RAND) {
         // no statistics
+    } else if (variant == METASD_PETC) {
+        petc_update(K, tau, *t, sa, sb, a, r);
     } else {
         int slot = *t % tau;
         wa[slot] = a;

@@ -390,7 +390,7 @@ __device__ void warp_bandit(const VerifyParams &p, int b, int t, int arm, double
     double *sa = p.st.stat_a + (size_t)b * K, *sb = p.st.stat_b + (size_t)b * K;
     int32_t *wa = p.st.win_arm + (size_t)b * tau;
     double *wr = p.st.win_reward + (size_t)b * tau;
-    if (p.bandit == METASD_EXP3 || p.bandit == METASD_RAND) {   // a draw, not an arg-max: one lane does it
+    if (p.bandit == METASD_EXP3 || p.bandit == METASD_RAND || p.bandit == METASD_PETC) {   // not an index arg-max: one lane does it
         if (lane == 0) {
             int32_t tt = t;
             bandit_update(p.bandit, K, p.gamma, tau, &tt, sa, sb, wa, wr, arm, r);

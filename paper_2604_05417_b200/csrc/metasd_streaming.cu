@@ -1041,7 +1041,7 @@ __global__ void reset_kernel(BanditState st, int max_batch, int K, int tau, int 
     const double first = variant == METASD_EXP3 ? 1.0 : 0.0;   // EXP3 starts from w(i) = 1
     for (int a = threadIdx.x; a < K; a += blockDim.x) {
         st.stat_a[(size_t)b * K + a] = first;
-        st.stat_b[(size_t)b * K + a] = 0.0;
+        st.stat_b[(size_t)b * K + a] = variant == METASD_PETC ? 1.0 : 0.0;   // PETC: every drafter starts in the set
     }
     for (int s = threadIdx.x; s < tau; s += blockDim.x) {
         st.win_arm[(size_t)b * tau + s] = 0;

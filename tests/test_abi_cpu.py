@@ -51,7 +51,7 @@ def test_host_side_validation(lib):
         bad.append((field, lib.metasd_init(C.byref(ctx), C.byref(cfg))))
         assert ctx.value is None
     assert all(code == M.ERR_INVALID_ARGUMENT for _, code in bad), bad
-    for field, value in [("logit_dtype", 7), ("bandit", 5), ("reward", 2), ("path", 9)]:
+    for field, value in [("logit_dtype", 7), ("bandit", 6), ("reward", 2), ("path", 9)]:
         cfg = M.default_config()
         setattr(cfg, field, value)
         assert lib.metasd_init(C.byref(ctx), C.byref(cfg)) == M.ERR_UNSUPPORTED

@@ -101,6 +101,17 @@ def test_randomised_policies(path, bandit):
 
 
 @pytest.mark.parametrize("path", PATHS)
+@pytest.mark.parametrize("N,budget", [(5, 30), (4, 16), (3, 2)])
+def test_pure_exploration_then_commit(path, N, budget):
+    """PETC: the Sequential Halving schedule, every halving and the committed drafter follow the oracle."""
+    from _harness import run_lockstep
+    sig = (0.3, 1.0, 2.0, 3.5, 0.6)[:N]
+    wl = base(B=7, N=N, k=3, V=2048, sigmas=sig).scaled(tau=budget)
+    c = report(run_lockstep(wl, rounds=budget + 12, path=path, bandit="petc", table_mode=True))
+    assert c["rounds"] == budget + 12 and c.get("near_tie_arm", 0) == 0
+
+
+@pytest.mark.parametrize("path", PATHS)
 def test_pointer_table_mode(path):
     """The kernel indexes a table of K drafter tensors and a [K,B,k] token table by arm."""
     from _harness import run_lockstep
