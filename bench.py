@@ -47,6 +47,9 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch (testing only)")
+    ap.add_argument("--k", type=int, default=0, help="override the workload's draft length (the N_max sweep)")
+    ap.add_argument("--ragged", action="store_true",
+                    help="per-sequence draft lengths, uniform in 1..k (seeded); bytes are counted per sequence")
     return ap.parse_args()
 
 
@@ -158,6 +161,8 @@ def main():
     wl = WORKLOADS[args.workload]
     if args.batch:
         wl = wl.scaled(B=args.batch)
+    if args.k:
+        wl = wl.scaled(k=args.k)
 
     if args.impl == "reference":
         return reference_arm(args, wl, rank)
@@ -184,6 +189,12 @@ def main():
         rd["table"] = M.pointer_table(rd["drafts"])
         rounds.append(rd)
     stride = wl.B * wl.k
+    lens = None
+    if args.ragged:
+        g = torch.Generator().manual_seed(4242 + rank)
+        lens = torch.randint(1, wl.k + 1, (wl.B,), generator=g, dtype=torch.int32)
+        lens_dev = lens.to(dev)
+        msd.set_draft_lengths(lens_dev)
     arm_buf = torch.empty(wl.B, dtype=torch.int32, device=dev)
     n_all = args.warmup + args.steps
     acc_all = torch.zeros((n_all, wl.B), dtype=torch.int32, device=dev)     # every step writes its own slice:
@@ -236,11 +247,13 @@ def main():
 
     # ---- roofline of the dominant kernel: algorithmic logit bytes of one round / its device time
     bytes_round = wl.bytes_per_round
+    if lens is not None:   # a sequence reads 2 k_b + 1 rows
+        bytes_round = int((2 * lens.to(torch.int64) + 1).sum().item()) * wl.V * (2 if wl.dtype == "bf16" else 4)
     kernel_ms = statistics.mean(step_ms)
     peak, peak_kind = measured_peak_gbs()
     achieved = bytes_round / (kernel_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": known_traffic(wl.name, path_name) if not args.batch else None, "peak_kind": "of " + peak_kind,
+                "traffic": known_traffic(wl.name, path_name) if not (args.batch or args.k or args.ragged) else None, "peak_kind": "of " + peak_kind,
                 "algorithmic_bytes_per_launch": bytes_round, "kernel_ms": kernel_ms,
                 "frac_of_8TBs_nominal": achieved / 8000.0,
                 "note": "duration = CUDA events around select+verify of one step (%s path)" % path_name}
@@ -251,6 +264,7 @@ def main():
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": wl.name, "B_per_gpu": wl.B, "N": wl.N, "k": wl.k, "V": wl.V, "logits": wl.dtype,
                    "temperature": wl.temperature, "bandit": wl.bandit, "path": path_name,
+                   "draft_len": "uniform 1..k per sequence" if args.ragged else "k for every sequence",
                    "l2": "inputs larger than L2: %.2f GB read per step, %d rotating input sets" % (bytes_round / 1e9, len(rounds))},
         "rounds_per_s": world * args.steps / (total_ms * 1e-3),
         "mean_accepted_len": tokens / (world * args.steps * wl.B) - 1.0,

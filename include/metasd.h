@@ -76,6 +76,7 @@ enum metasd_path {
 #define METASD_STATUS_TOKEN_OOR 2u /* a drafted token id was outside [0, V) */
 #define METASD_STATUS_Q_ZERO    4u /* the drafter gave probability 0 to its own drafted token */
 #define METASD_STATUS_TIMEOUT   8u /* a bounded wait on an asynchronous copy ran out: outputs of that call are undefined */
+#define METASD_STATUS_BAD_LENGTH 32u /* a registered per-sequence draft length was outside 1 .. k: it was clamped */
 #define METASD_STATUS_BAD_POINTER 16u /* the drafter table of a call held a NULL or misaligned entry: its rows are never
                                         read and the outputs of the sequences that played that drafter are meaningless */
 
@@ -163,6 +164,16 @@ int metasd_verify(metasd_ctx *ctx, int32_t batch, int32_t k, const void *target_
                   const int32_t *draft_tokens, int64_t token_arm_stride, float temperature,
                   uint64_t seed, int32_t *accepted_len, int32_t *next_token, float *reward,
                   metasd_diag *diag, void *stream);
+
+/* Per-sequence draft lengths (the paper fixes N_max per run and sweeps it as an ablation; a serving batch mixes
+ * lengths): draft_len is a DEVICE array [max_batch] of int32 that metasd_verify reads on every later call, or NULL
+ * to go back to "every sequence drafted k tokens".  Sequence b then uses target rows 0 .. draft_len[b] (the last one
+ * is its bonus row) and draft rows / tokens 0 .. draft_len[b]-1 of its k-padded slots; nothing behind them is read,
+ * accepted_len[b] <= draft_len[b], and both rewards are normalised by draft_len[b].  The layout of every buffer is
+ * unchanged.  A length outside 1 .. k is clamped and sets METASD_STATUS_BAD_LENGTH.  The caller owns the array and
+ * keeps it valid (its contents may change between calls, in stream order).  Streaming path only: with lengths
+ * registered, a context whose path is METASD_PATH_FUSED returns METASD_ERR_UNSUPPORTED from metasd_verify. */
+int metasd_set_draft_lengths(metasd_ctx *ctx, const int32_t *draft_len);
 
 /* The same round with HOST buffers (gathered draft logits only): copies the inputs to the context's
  * staging memory, runs metasd_verify, copies the three outputs (and host_arm_next, optional: the

@@ -498,10 +498,12 @@ void msdo_bandit_update(int variant, int K, double gamma, int tau, int32_t *t, d
 
 /* One verification round for a batch.  draft_gathered: [B,k,V] already gathered
  * by arm, or NULL with drafter_tables[K] (each [B,k,V]) indexed by arm[b].
+ * draft_len: NULL, or [B] drafted tokens per sequence this round (1..k).
  * rounds[b] = the sequence's round counter t (keys the uniforms);
  * sequence_base + b = the sequence id in the key. */
 void msdo_verify_batch(int B, int k, int V, int dtype, const void *target, const void *draft_gathered,
                        const void *const *drafter_tables, const int32_t *arm, const int32_t *tokens,
+                       const int32_t *draft_len,
                        double temperature, double reward_temperature, int reward_kind, uint64_t seed,
                        uint32_t sequence_base, const int32_t *rounds, int32_t *accepted_len,
                        int32_t *next_token, double *reward, double *p_x, double *q_x, double *D,
@@ -514,18 +516,24 @@ void msdo_verify_batch(int B, int k, int V, int dtype, const void *target, const
         double *draft_rows = rows + (size_t)(k + 1) * V;
         double *scratch = draft_rows + (size_t)k * V;
         const void *draft_base = draft_gathered ? draft_gathered : drafter_tables[arm[b]];
-        for (int j = 0; j <= k; ++j)
+        /* A sequence that drafted kb <= k tokens this round is a round of draft length kb on the first kb + 1
+         * target rows and kb draft rows of its (k-padded) slots; whatever lies behind them is not looked at.
+         * Lengths outside 1..k are clamped (the caller's library flags them). */
+        int kb = draft_len ? draft_len[b] : k;
+        if (kb < 1) kb = 1;
+        if (kb > k) kb = k;
+        for (int j = 0; j <= kb; ++j)
             msdo_load_row(target, dtype, ((size_t)b * (k + 1) + j) * V, V, target_rows + (size_t)j * V);
-        for (int j = 0; j < k; ++j)
+        for (int j = 0; j < kb; ++j)
             msdo_load_row(draft_base, dtype, ((size_t)b * k + j) * V, V, draft_rows + (size_t)j * V);
         double u_accept[64], u_sample[65];
-        for (int j = 0; j <= k; ++j) {
+        for (int j = 0; j <= kb; ++j) {
             double ua, us;
             msdo_round_uniforms(seed, sequence_base + (uint32_t)b, (uint32_t)rounds[b], (uint32_t)j, &ua, &us);
-            if (j < k) { u_accept[j] = ua; u_accept_out[(size_t)b * k + j] = ua; }
+            if (j < kb) { u_accept[j] = ua; u_accept_out[(size_t)b * k + j] = ua; }
             u_sample[j] = us;
         }
-        msdo_verify_sequence(target_rows, draft_rows, tokens + (size_t)b * k, k, V, temperature,
+        msdo_verify_sequence(target_rows, draft_rows, tokens + (size_t)b * k, kb, V, temperature,
                              reward_temperature, reward_kind, u_accept, u_sample, accepted_len + b,
                              next_token + b, reward + b, p_x + (size_t)b * k, q_x + (size_t)b * k,
                              D + (size_t)b * k, accept + (size_t)b * k, sample_margin + b, status + b,

@@ -221,7 +221,7 @@ class OracleMetaSD:
         return arm
 
     def verify(self, target_logits, draft_logits, draft_tokens, temperature, seed,
-               drafter_tables=None, update=True):
+               drafter_tables=None, update=True, draft_len=None):
         """One round.  draft_logits: [B,k,V] gathered by arm, or None with
         drafter_tables = list of K [B,k,V] tensors (indexed by this oracle's own arm)."""
         c = self.cfg
@@ -246,6 +246,7 @@ class OracleMetaSD:
             arr = (C.c_void_p * len(tabs))(*[t_.ctypes.data for t_ in tabs])
             d_ptr, tab_ptr = None, arr
         tok = np.ascontiguousarray(np.asarray(draft_tokens, dtype=np.int32)).reshape(B, k)
+        lens = None if draft_len is None else np.ascontiguousarray(np.asarray(draft_len, dtype=np.int32)).reshape(B)
         out = dict(
             arm=arm,
             accepted_len=np.zeros(B, dtype=np.int32), next_token=np.zeros(B, dtype=np.int32),
@@ -255,7 +256,7 @@ class OracleMetaSD:
             round=self.t[:B].copy())
         lib().msdo_verify_batch(
             C.c_int(B), C.c_int(k), C.c_int(V), C.c_int(dtype), _p(tgt), d_ptr, tab_ptr, _p(arm),
-            _p(tok), C.c_double(temperature), C.c_double(c.reward_temperature), C.c_int(c.reward),
+            _p(tok), None if lens is None else _p(lens), C.c_double(temperature), C.c_double(c.reward_temperature), C.c_int(c.reward),
             C.c_uint64(seed), C.c_uint32(c.sequence_base), _p(self.t), _p(out["accepted_len"]),
             _p(out["next_token"]), _p(out["reward"]), _p(out["p_x"]), _p(out["q_x"]), _p(out["D"]),
             _p(out["accept"]), _p(out["u_accept"]), _p(out["sample_margin"]), _p(out["status"]))

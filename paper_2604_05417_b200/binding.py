@@ -20,7 +20,7 @@ BF16, FP32 = 0, 1
 UCB, DUCB, SWUCB, EXP3, RAND, PETC = 0, 1, 2, 3, 4, 5
 REWARD_BD, REWARD_BE = 0, 1
 PATH_AUTO, PATH_STREAMING, PATH_FUSED = 0, 1, 2
-STATUS_NONFINITE, STATUS_TOKEN_OOR, STATUS_Q_ZERO, STATUS_TIMEOUT, STATUS_BAD_POINTER = 1, 2, 4, 8, 16
+STATUS_NONFINITE, STATUS_TOKEN_OOR, STATUS_Q_ZERO, STATUS_TIMEOUT, STATUS_BAD_POINTER, STATUS_BAD_LENGTH = 1, 2, 4, 8, 16, 32
 
 OK, ERR_INVALID_ARGUMENT, ERR_UNSUPPORTED, ERR_CUDA, ERR_NO_MEMORY, ERR_BAD_STATE_BLOB = 0, -1, -2, -3, -4, -5
 
@@ -31,7 +31,7 @@ EXPORTS = (
     "metasd_default_config", "metasd_init", "metasd_destroy", "metasd_reset", "metasd_select",
     "metasd_verify", "metasd_verify_host", "metasd_state_bytes", "metasd_state_export",
     "metasd_state_import", "metasd_last_status", "metasd_kernel_launches", "metasd_resolved_path",
-    "metasd_strerror", "metasd_verify_noalloc",
+    "metasd_strerror", "metasd_verify_noalloc", "metasd_set_draft_lengths",
 )
 
 
@@ -88,6 +88,7 @@ def load_library(path: Optional[str] = None):
     lib.metasd_state_import.argtypes = [vp, vp, C.c_size_t, vp]
     lib.metasd_last_status.argtypes = [vp, C.POINTER(C.c_uint32), vp]
     lib.metasd_kernel_launches.argtypes = [vp]
+    lib.metasd_set_draft_lengths.argtypes = [vp, vp]
     lib.metasd_kernel_launches.restype = u64
     lib.metasd_resolved_path.argtypes = [vp, i32]
     lib.metasd_verify_noalloc.argtypes = [i32, i32, i32, i32, vp, vp, vp, C.c_float, C.c_float, i32, u64, C.c_uint32,
@@ -223,6 +224,16 @@ class MetaSD:
     def state_import(self, blob: bytes):
         buf = C.create_string_buffer(blob, len(blob))
         _check(self.lib.metasd_state_import(self._ctx, buf, len(blob), _stream(self.device)), "metasd_state_import")
+
+    def set_draft_lengths(self, draft_len: Optional[torch.Tensor]):
+        """Registers an int32 device tensor [max_batch] of per-sequence draft lengths (None: all sequences draft k).
+        The tensor is kept alive by this object and read by every later verify call."""
+        if draft_len is not None:
+            assert draft_len.dtype == torch.int32 and draft_len.is_cuda and draft_len.is_contiguous()
+            assert draft_len.numel() >= self.cfg.max_batch
+        self._draft_len = draft_len
+        _check(self.lib.metasd_set_draft_lengths(self._ctx, None if draft_len is None else draft_len.data_ptr()),
+               "metasd_set_draft_lengths")
 
     def last_status(self) -> int:
         flags = C.c_uint32()

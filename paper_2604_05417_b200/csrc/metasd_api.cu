@@ -16,6 +16,7 @@ struct metasd_ctx {
     RowStats *stats;     // scratch of the streaming path: [max_batch, max_draft + 1]
     uint32_t *status;    // device status word
     const void **table_clean;   // the checked copy of the caller's drafter table (16 entries)
+    const int32_t *draft_len;   // the caller's per-sequence draft lengths (device), or nullptr
     uint64_t launches;
     // staging for metasd_verify_host
     void *stage_target, *stage_draft;
@@ -235,6 +236,7 @@ int metasd_verify(metasd_ctx *ctx, int32_t batch, int32_t k, const void *target_
     p.sequence_base = cfg.sequence_base;
     p.target = target_logits; p.draft = draft_logits; p.drafter_ptrs = drafter_ptrs;
     p.tokens = draft_tokens; p.token_arm_stride = token_arm_stride;
+    p.draft_len = ctx->draft_len;
     p.greedy = temperature == 0.f;
     const double T = p.greedy ? cfg.reward_temperature : (double)temperature;
     p.c = (float)(1.4426950408889634 / T);
@@ -260,6 +262,7 @@ int metasd_verify(metasd_ctx *ctx, int32_t batch, int32_t k, const void *target_
         ctx->launches += 1;
         p.drafter_ptrs = ctx->table_clean;
     }
+    if (ctx->draft_len && cfg.path == METASD_PATH_FUSED) return METASD_ERR_UNSUPPORTED;
     if (metasd_resolved_path(ctx, k) == METASD_PATH_FUSED && p.vector_ok)
         e = launch_fused(p, cfg.logit_dtype, ctx->plan, (cudaStream_t)stream, &ctx->launches);
     else if (cfg.path == METASD_PATH_FUSED)
@@ -267,6 +270,13 @@ int metasd_verify(metasd_ctx *ctx, int32_t batch, int32_t k, const void *target_
     else
         e = launch_streaming(p, cfg.logit_dtype, (cudaStream_t)stream, &ctx->launches);
     return e == cudaSuccess ? METASD_OK : cuda_fail(e);
+}
+
+int metasd_set_draft_lengths(metasd_ctx *ctx, const int32_t *draft_len)
+{
+    if (!ctx) return METASD_ERR_INVALID_ARGUMENT;
+    ctx->draft_len = draft_len;
+    return METASD_OK;
 }
 
 int metasd_verify_host(metasd_ctx *ctx, int32_t batch, int32_t k, const void *host_target_logits,

@@ -84,6 +84,15 @@ template <> struct Logit<float> {
     __device__ static __forceinline__ float scalar(const float *p, size_t i) { return p[i]; }
 };
 
+// Tokens sequence b drafted this round: the call's k unless the caller registered per-sequence lengths, which are
+// clamped to 1 .. k (the epilogue flags a length outside that range).
+__device__ __forceinline__ int drafted(const int32_t *draft_len, int b, int k)
+{
+    if (!draft_len) return k;
+    const int kb = draft_len[b];
+    return kb < 1 ? 1 : (kb > k ? k : kb);
+}
+
 // Streaming 16-byte load that does not allocate in L1.
 __device__ __forceinline__ uint4 ld_stream(const void *p)
 {

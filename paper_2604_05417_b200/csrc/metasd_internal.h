@@ -45,6 +45,7 @@ struct VerifyParams {
     const void *draft;                 // gathered, or nullptr
     const void *const *drafter_ptrs;   // table, or nullptr
     const int32_t *tokens;
+    const int32_t *draft_len;          // [batch] tokens drafted per sequence this round, or nullptr = k for all
     int64_t token_arm_stride;
     // math
     float c;           // log2(e) / softmax temperature

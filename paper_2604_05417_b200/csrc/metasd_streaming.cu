@@ -40,7 +40,9 @@ __global__ void __launch_bounds__(K1_THREADS) row_stats_kernel(const VerifyParam
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int V = p.V;
     const float c = p.c;
-    const bool pair = j < p.k;
+    const int kb = drafted(p.draft_len, b, p.k);
+    if (j > kb) return;   // behind this sequence's bonus row: nothing to read
+    const bool pair = j < kb;
 
     const LT *a = reinterpret_cast<const LT *>(p.target) + ((size_t)b * (p.k + 1) + j) * V;
     const LT *d = pair ? draft_rows<LT>(p, b) + ((size_t)b * p.k + j) * V : nullptr;
@@ -195,7 +197,9 @@ __global__ void __launch_bounds__(THREADS, MINB) row_stats_staged_kernel(const V
     const int j = blockIdx.x, b = blockIdx.y;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const float c = p.c;
-    const bool pair = j < p.k;
+    const int kb = drafted(p.draft_len, b, p.k);
+    if (j > kb) return;   // behind this sequence's bonus row: nothing to read
+    const bool pair = j < kb;
 
     const uint4 *a4 = reinterpret_cast<const uint4 *>(reinterpret_cast<const LT *>(p.target) + ((size_t)b * (p.k + 1) + j) * p.V);
     const uint4 *d4 = pair ? reinterpret_cast<const uint4 *>(draft_rows<LT>(p, b) + ((size_t)b * p.k + j) * p.V) : nullptr;
@@ -800,11 +804,12 @@ template <typename LT, bool VECTOR, int K2_THREADS>
 __global__ void __launch_bounds__(K2_THREADS, 1024 / K2_THREADS) epilogue_kernel(const VerifyParams p)
 {
     const int b = blockIdx.x, tid = threadIdx.x;
-    const int k = p.k, V = p.V, K = p.K;
+    const int k_slots = p.k, V = p.V, K = p.K;   // rows and tokens are laid out for k_slots positions per sequence
+    const int k = drafted(p.draft_len, b, k_slots);   // positions this sequence drafted this round
     const float c = p.c;
-    const LT *target = reinterpret_cast<const LT *>(p.target) + (size_t)b * (k + 1) * V;
-    const LT *draft = draft_rows<LT>(p, b) + (size_t)b * k * V;
-    const RowStats *stats = p.stats + (size_t)b * (k + 1);
+    const LT *target = reinterpret_cast<const LT *>(p.target) + (size_t)b * (k_slots + 1) * V;
+    const LT *draft = draft_rows<LT>(p, b) + (size_t)b * k_slots * V;
+    const RowStats *stats = p.stats + (size_t)b * (k_slots + 1);
 
     __shared__ int sh_nacc, sh_mode, sh_tok;
     __shared__ float sh_u;
@@ -814,14 +819,14 @@ __global__ void __launch_bounds__(K2_THREADS, 1024 / K2_THREADS) epilogue_kernel
     __shared__ int sh_accept[16];
     __shared__ double sh_align[16];
 
-    if (tid == 0) sh_flags = 0;
+    if (tid == 0) sh_flags = (p.draft_len && p.draft_len[b] != k) ? METASD_STATUS_BAD_LENGTH : 0u;
     __syncthreads();
     const int t = p.st.t[b];
     const int arm = p.st.arm[b];
     if (tid < k) {
         // position j = tid: the accept test of Algorithm 4
         const int j = tid;
-        const int32_t *tokens = p.tokens + (p.token_arm_stride ? (size_t)arm * p.token_arm_stride : 0) + (size_t)b * k;
+        const int32_t *tokens = p.tokens + (p.token_arm_stride ? (size_t)arm * p.token_arm_stride : 0) + (size_t)b * k_slots;
         const RowStats r = stats[j];
         const uint4 words = round_words(p.seed, p.sequence_base + (uint32_t)b, (uint32_t)t, (uint32_t)j);
         const float u = uniform24(words.x);
@@ -853,7 +858,7 @@ __global__ void __launch_bounds__(K2_THREADS, 1024 / K2_THREADS) epilogue_kernel
         if (p.diag) {
             metasd_diag dg;
             dg.p_x = p_x; dg.q_x = q_x; dg.D = D; dg.u = u; dg.accept = accepted ? 1 : 0;
-            p.diag[(size_t)b * k + j] = dg;
+            p.diag[(size_t)b * k_slots + j] = dg;
         }
     }
     __syncthreads();
@@ -921,7 +926,7 @@ static cudaError_t launch_streaming_t(const VerifyParams &p, cudaStream_t stream
 {
     dim3 g1(p.k + 1, p.batch);
     const bool big_ctas = p.batch <= 320;   // up to about two sequences per SM
-    if (p.vector_ok && p.grp_size > 1) {
+    if (p.vector_ok && p.grp_size > 1 && !p.draft_len) {
         const int n_items = p.batch * (p.k + 1);
         int n_groups = p.grp_ctas / p.grp_size;
         if (n_groups > n_items) n_groups = n_items;

@@ -148,6 +148,82 @@ def test_batch_shard_uses_global_sequence_ids(path):
         m.close()
 
 
+@pytest.mark.parametrize("T", [1.0, 0.0])
+@pytest.mark.parametrize("dtype", ["bf16", "fp32"])
+def test_per_sequence_draft_lengths(T, dtype):
+    """Sequences that drafted fewer than k tokens: only their own rows are read (the rest is poisoned with NaN),
+    accepted lengths, tokens, rewards and the bandit follow the oracle's ragged round."""
+    from _harness import make_pair, TOL, NEAR
+    wl = base(B=11, N=3, k=5, V=4096 + 8, sigmas=(0.4, 1.2, 2.5)).scaled(dtype=dtype, temperature=T)
+    dev = torch.device("cuda", 0)
+    gen = RoundGenerator(wl, device=dev, seed=11)
+    gpu, orc = make_pair(wl, path=M.PATH_STREAMING)
+    rng = np.random.RandomState(2)
+    lens_dev = torch.zeros(wl.B, dtype=torch.int32, device=dev)
+    gpu.set_draft_lengths(lens_dev)
+    try:
+        for t in range(8):
+            lens = rng.randint(1, wl.k + 1, size=wl.B).astype(np.int32)
+            if t == 0:
+                lens[:] = wl.k
+            lens_dev.copy_(torch.from_numpy(lens))
+            arm = orc.select()
+            assert np.array_equal(gpu.select().cpu().numpy(), arm)
+            rd = gen.gathered_round(t, arm)
+            target, draft = rd["target"].clone(), rd["draft"].clone()
+            for b in range(wl.B):
+                target[b, lens[b] + 1:] = float("nan")
+                draft[b, lens[b]:] = float("nan")
+            res = gpu.verify(target, draft, rd["tokens"], T, 99, want_diag=True)
+            out = orc.verify(target, draft, rd["tokens"].cpu().numpy(), T, 99, draft_len=lens)
+            assert gpu.last_status() == 0 and (out["status"] == 0).all()
+            g_len = res.accepted_len.cpu().numpy()
+            assert np.array_equal(g_len, out["accepted_len"]) and (g_len <= lens).all()
+            g_tok = res.next_token.cpu().numpy()
+            firm = out["sample_margin"] > NEAR if T > 0 else np.ones(wl.B, dtype=bool)
+            assert np.array_equal(g_tok[firm], out["next_token"][firm])
+            np.testing.assert_allclose(res.reward.cpu().numpy(), out["reward"], rtol=0, atol=TOL)
+            D = res.diag_fields()[2].cpu().numpy()
+            for b in range(wl.B):
+                np.testing.assert_allclose(D[b, :lens[b]], out["D"][b, :lens[b]], rtol=0, atol=TOL)
+        st = M.parse_state(gpu.state_export(), wl.B, wl.N, wl.tau)
+        assert np.array_equal(st["t"], orc.t)
+        np.testing.assert_allclose(st["stat_a"], orc.stat_a, rtol=0, atol=1e-5)
+        # lengths outside 1 .. k are clamped and flagged; clearing the registration restores the fixed length
+        lens_dev.copy_(torch.tensor([0, wl.k + 7] + [2] * (wl.B - 2), dtype=torch.int32))
+        arm = orc.select()
+        rd = gen.gathered_round(8, arm)
+        res = gpu.verify(rd["target"], rd["draft"], rd["tokens"], T, 99)
+        out = orc.verify(rd["target"], rd["draft"], rd["tokens"].cpu().numpy(), T, 99,
+                         draft_len=np.array([1, wl.k] + [2] * (wl.B - 2)))
+        assert gpu.last_status() == M.STATUS_BAD_LENGTH
+        assert np.array_equal(res.accepted_len.cpu().numpy(), out["accepted_len"])
+        gpu.set_draft_lengths(None)
+        arm = orc.select()
+        rd = gen.gathered_round(9, arm)
+        res = gpu.verify(rd["target"], rd["draft"], rd["tokens"], T, 99)
+        out = orc.verify(rd["target"], rd["draft"], rd["tokens"].cpu().numpy(), T, 99)
+        assert gpu.last_status() == 0
+        assert np.array_equal(res.accepted_len.cpu().numpy(), out["accepted_len"])
+    finally:
+        gpu.close()
+
+
+def test_fused_path_declines_per_sequence_draft_lengths():
+    from _harness import new_context
+    gpu = new_context(4, 2, 3, 4096, path=M.PATH_FUSED)
+    dev = torch.device("cuda", 0)
+    try:
+        gpu.set_draft_lengths(torch.full((4,), 2, dtype=torch.int32, device=dev))
+        wl = base(B=4, N=2, k=3, V=4096, sigmas=(0.5, 2.0))
+        rd = RoundGenerator(wl, device=dev, seed=1).gathered_round(0, np.zeros(4, dtype=np.int64))
+        with pytest.raises(M.MetasdError) as err:
+            gpu.verify(rd["target"], rd["draft"], rd["tokens"], 1.0, 5)
+        assert err.value.code == M.ERR_UNSUPPORTED
+    finally:
+        gpu.close()
+
+
 @pytest.mark.parametrize("path", PATHS)
 def test_defined_outcomes_of_anomalous_inputs(path):
     """NaN rows, masked (-inf) logits, out-of-range tokens: same defined outputs and status bits."""

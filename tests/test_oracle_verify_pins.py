@@ -488,3 +488,36 @@ def test_single_drafter_stopping_time_bounds():
     assert B_tok * scale - 1 - 4 * se < tau.mean() <= (B_tok + 1) * scale + 4 * se
     # tokens out = rounds + accepted tokens (proof of the stopping-time lemma), per sequence
     assert (length >= B_tok).all() and (length < B_tok + k + 1).all()
+
+
+def test_ragged_round_equals_the_fixed_length_round_on_the_truncated_rows():
+    """A sequence that drafted kb < k tokens is a round of draft length kb on its first kb + 1 target rows and
+    kb draft rows: same uniforms (keyed by position), reward normalised by kb, nothing behind those rows is read."""
+    rng = np.random.RandomState(5)
+    B, k, V = 6, 5, 97
+    target = rng.randn(B, k + 1, V).astype(np.float32) * 2
+    draft = (target[:, :k] + rng.randn(B, k, V).astype(np.float32)).astype(np.float32)
+    tokens = rng.randint(0, V, size=(B, k)).astype(np.int32)
+    lens = np.array([1, 2, 3, 4, 5, 3], dtype=np.int32)
+    poisoned_t, poisoned_d = target.copy(), draft.copy()
+    for b in range(B):                                   # rows behind the drafted ones must not matter
+        poisoned_t[b, lens[b] + 1:] = np.nan
+        poisoned_d[b, lens[b]:] = np.nan
+    for reward in (O.REWARD_BD, O.REWARD_BE):
+        cfg = O.OracleConfig(max_batch=B, n_drafters=2, vocab=V, reward=reward)
+        ragged = O.OracleMetaSD(cfg).verify(poisoned_t, poisoned_d, tokens, 1.0, 77, update=False, draft_len=lens)
+        assert (ragged["status"] == 0).all()
+        for b in range(B):
+            kb = int(lens[b])
+            one = O.OracleMetaSD(O.OracleConfig(max_batch=1, n_drafters=2, vocab=V, reward=reward, sequence_base=b))
+            fixed = one.verify(target[b:b + 1, :kb + 1], draft[b:b + 1, :kb], tokens[b:b + 1, :kb], 1.0, 77,
+                               update=False)
+            assert ragged["accepted_len"][b] == fixed["accepted_len"][0] <= kb
+            assert ragged["next_token"][b] == fixed["next_token"][0]
+            assert ragged["reward"][b] == fixed["reward"][0]
+            assert np.array_equal(ragged["D"][b, :kb], fixed["D"][0])
+            assert np.array_equal(ragged["accept"][b, :kb], fixed["accept"][0])
+    full = O.OracleMetaSD(cfg).verify(target, draft, tokens, 1.0, 77, update=False, draft_len=np.full(B, k))
+    plain = O.OracleMetaSD(cfg).verify(target, draft, tokens, 1.0, 77, update=False)
+    for key in ("accepted_len", "next_token", "reward", "D", "accept"):
+        assert np.array_equal(full[key], plain[key])
