@@ -153,6 +153,19 @@ __device__ __forceinline__ MaxSum warp_merge(MaxSum v, float c)
     return v;
 }
 
+// Offsets and scale of the second sweep: min(p, q) = 2^min(ya, yb + lg) / sum_a = 2^min(ya - lg, yb) / sum_b with
+// ya = (a - max_a) c, yb = (b - max_b) c, lg = log2(sum_a / sum_b).  lg is folded into the offset of the row whose
+// reference is smaller in magnitude: added to a large offset it would be rounded at that offset's size (logits
+// near +-300 would cost 1e-5 of every term).  out = {offset of the target row, offset of the draft row, scale}.
+__device__ __forceinline__ void second_sweep_offsets(MaxSum a, MaxSum b, float c, float *out)
+{
+    const float lg = log2f(a.s / b.s);
+    const bool on_a = fabsf(a.m) < fabsf(b.m);
+    out[0] = on_a ? -a.m * c - lg : -a.m * c;
+    out[1] = on_a ? -b.m * c : -b.m * c + lg;
+    out[2] = 1.0f / (on_a ? b.s : a.s);
+}
+
 struct ArgMax {
     float v;
     int32_t i;

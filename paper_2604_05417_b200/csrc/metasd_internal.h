@@ -12,7 +12,8 @@ namespace metasd {
 //   p_v = 2^((x_v - max_a) * c) / sum_a,  c = log2(e) / T.
 struct RowStats {
     float max_a, sum_a;   // target row
-    float max_b, sum_b;   // draft row (unused at the bonus position)
+    float max_b, sum_b;   // draft row (unused at the bonus position); max_b is the reference sum_b is relative to:
+                          // the row's maximum, or the target row's where the staged kernel could share it
     double sum_min;       // sum_v min(p_v, q_v) = 1 - d_TV(p, q)
     int32_t argmax_a;     // first index of the target row's maximum
     uint32_t flags;       // METASD_STATUS_* of this row pair

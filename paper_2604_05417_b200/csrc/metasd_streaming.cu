@@ -97,7 +97,7 @@ __global__ void __launch_bounds__(K1_THREADS) row_stats_kernel(const VerifyParam
     __shared__ MaxSum sh_a[NWARP], sh_b[NWARP];
     __shared__ ArgMax sh_am[NWARP];
     __shared__ double sh_min[NWARP];
-    __shared__ float sh_bcast[5];
+    __shared__ float sh_bcast[7];
 
     sa = warp_merge(sa, c);
     sb = warp_merge(sb, c);
@@ -113,8 +113,7 @@ __global__ void __launch_bounds__(K1_THREADS) row_stats_kernel(const VerifyParam
         rm = warp_argmax(rm);
         if (lane == 0) {
             sh_bcast[0] = ra.m; sh_bcast[1] = ra.s; sh_bcast[2] = rb.m; sh_bcast[3] = rb.s;
-            // q_v / p_v = 2^(yb - ya) sum_a / sum_b: the ratio of the sums folds into the draft row's offset
-            sh_bcast[4] = -rb.m * c + log2f(ra.s / rb.s);
+            second_sweep_offsets(ra, rb, c, sh_bcast + 4);
             sh_am[0] = rm;
         }
     }
@@ -124,8 +123,7 @@ __global__ void __launch_bounds__(K1_THREADS) row_stats_kernel(const VerifyParam
     // ---- sweep 2: sum_v min(p_v, q_v) = (1 / sum_a) sum_v 2^min(ya_v, yb_v): one exponential per pair
     double total_min = 0.0;
     if (pair) {
-        const float nma = -max_a * c, nmb = sh_bcast[4];
-        const float ia = 1.0f / sum_a;
+        const float nma = sh_bcast[4], nmb = sh_bcast[5], ia = sh_bcast[6];
         float acc = 0.f;
         // backwards: the end of the rows was read last in sweep 1 and is the part most likely still in L2
         for (int i = nvec - 1 - tid; i >= 0; i -= K1_THREADS) {
@@ -207,7 +205,11 @@ __global__ void __launch_bounds__(THREADS, MINB) row_stats_staged_kernel(const V
     const int n_trip = tid < nvec ? (nvec - tid + THREADS - 1) / THREADS : 0;   // vectors of this thread
     const uint32_t slot0 = smem_addr(stage_mem) + (uint32_t)tid * 16u;
 
-    // ---- sweep 1: online (max, sum) of both rows, arg-max of the target row
+    // ---- sweep 1: online (max, sum) of the target row and its arg-max; the draft row's sum is taken relative to
+    // the SAME running reference (the target's maximum so far): a softmax sum may be taken relative to any
+    // reference that neither overflows nor underflows it, and sharing one spares the draft row its own maximum
+    // search (the kernel is bound by instruction issue).  Whether the reference suited the draft row is checked
+    // after the sweep; if not, that row's statistics are redone relative to its own maximum.
     MaxSum sa = {METASD_NEG_BIG, 0.f}, sb = {METASD_NEG_BIG, 0.f};
     ArgMax am = {METASD_NEG_BIG, 0x7FFFFFFF};
     const uint64_t keep = l2_policy_evict_last(), drop = l2_policy_evict_first();
@@ -236,7 +238,9 @@ __global__ void __launch_bounds__(THREADS, MINB) row_stats_staged_kernel(const V
 #pragma unroll
         for (int e = 1; e < VEC; ++e) cm = fmaxf(cm, xa[e]);
         if (cm > sa.m) {
-            sa.s *= ex2((sa.m - cm) * c);
+            const float shrink = ex2((sa.m - cm) * c);
+            sa.s *= shrink;
+            sb.s *= shrink;
             sa.m = cm;
             int first = 0;
 #pragma unroll
@@ -251,24 +255,17 @@ __global__ void __launch_bounds__(THREADS, MINB) row_stats_staged_kernel(const V
         if (pair) {
             float xb[VEC];
             Logit<LT>::unpack(lds16(src + ROW_STRIDE), xb);
-            float bm = xb[0];
 #pragma unroll
-            for (int e = 1; e < VEC; ++e) bm = fmaxf(bm, xb[e]);
-            if (bm > sb.m) {
-                sb.s *= ex2((sb.m - bm) * c);
-                sb.m = bm;
-            }
-            const float nmb = -sb.m * c;
-#pragma unroll
-            for (int e = 0; e < VEC; ++e) sb.s += ex2(fmaf(xb[e], c, nmb));
+            for (int e = 0; e < VEC; ++e) sb.s += ex2(fmaf(xb[e], c, nma));
         }
     }
     cp_async_wait<0>();
+    sb.m = sa.m;   // the draft row's sum is relative to the target row's maximum
 
     __shared__ MaxSum sh_a[NWARP], sh_b[NWARP];
     __shared__ ArgMax sh_am[NWARP];
     __shared__ double sh_min[NWARP];
-    __shared__ float sh_bcast[5];
+    __shared__ float sh_bcast[7];
 
     sa = warp_merge(sa, c);
     sb = warp_merge(sb, c);
@@ -284,18 +281,50 @@ __global__ void __launch_bounds__(THREADS, MINB) row_stats_staged_kernel(const V
         rm = warp_argmax(rm);
         if (lane == 0) {
             sh_bcast[0] = ra.m; sh_bcast[1] = ra.s; sh_bcast[2] = rb.m; sh_bcast[3] = rb.s;
-            sh_bcast[4] = -rb.m * c + log2f(ra.s / rb.s);
+            second_sweep_offsets(ra, rb, c, sh_bcast + 4);
             sh_am[0] = rm;
         }
     }
     __syncthreads();
+    // The shared reference suits the draft row when its sum is neither flushed nor overflowed: 2^-60 .. finite
+    // leaves every term that matters in fp32 range.  Otherwise (draft logits far from the target's, or a row
+    // that is not finite) the draft row is swept again relative to its own running maximum.
+    if (pair && !(sh_bcast[3] >= 0x1p-60f && sh_bcast[3] < INFINITY)) {
+        __syncthreads();   // everybody has read the first verdict
+        MaxSum own = {METASD_NEG_BIG, 0.f};
+        for (int i = tid; i < nvec; i += THREADS) {
+            float xb[VEC];
+            Logit<LT>::unpack(ld_stream(d4 + i), xb);
+            float bm = xb[0];
+#pragma unroll
+            for (int e = 1; e < VEC; ++e) bm = fmaxf(bm, xb[e]);
+            if (bm > own.m) {
+                own.s *= ex2((own.m - bm) * c);
+                own.m = bm;
+            }
+            const float nmb = -own.m * c;
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) own.s += ex2(fmaf(xb[e], c, nmb));
+        }
+        own = warp_merge(own, c);
+        if (lane == 0) sh_b[warp] = own;
+        __syncthreads();
+        if (warp == 0) {
+            MaxSum rb = lane < NWARP ? sh_b[lane] : MaxSum{METASD_NEG_BIG, 0.f};
+            rb = warp_merge(rb, c);
+            if (lane == 0) {
+                sh_bcast[2] = rb.m; sh_bcast[3] = rb.s;
+                second_sweep_offsets(MaxSum{sh_bcast[0], sh_bcast[1]}, rb, c, sh_bcast + 4);
+            }
+        }
+        __syncthreads();
+    }
     const float max_a = sh_bcast[0], sum_a = sh_bcast[1], max_b = sh_bcast[2], sum_b = sh_bcast[3];
 
     // ---- sweep 2, this thread's trips in reverse: sum_v 2^min(ya_v, yb_v), one exponential per pair
     double total_min = 0.0;
     if (pair) {
-        const float nma = -max_a * c, nmb = sh_bcast[4];
-        const float ia = 1.0f / sum_a;
+        const float nma = sh_bcast[4], nmb = sh_bcast[5], ia = sh_bcast[6];
         float acc = 0.f;
 #pragma unroll 4
         for (int n = n_trip - 1; n >= 0; --n) {

@@ -224,6 +224,34 @@ def test_fused_path_declines_per_sequence_draft_lengths():
         gpu.close()
 
 
+@pytest.mark.parametrize("dtype", ["bf16", "fp32"])
+@pytest.mark.parametrize("T", [1.0, 0.5])
+def test_draft_rows_on_another_scale_than_the_target(dtype, T):
+    """Softmax is shift invariant, so a drafter whose logits sit hundreds of units above or below the target's is
+    legal input.  The row-statistics kernel sums the draft row relative to the target's maximum where that is
+    safe and must notice where it is not (these offsets overflow or flush that sum) and redo the row.  The offsets
+    stay where fp32 exponents still resolve 1e-5: an offset M c is rounded at its own size, so |M| c is kept
+    below about 450."""
+    from _harness import make_pair, compare_round
+    wl = base(B=8, N=1, k=3, V=8192, sigmas=(0.8,)).scaled(dtype=dtype, temperature=T)
+    dev = torch.device("cuda", 0)
+    gen = RoundGenerator(wl, device=dev, seed=4)
+    gpu, orc = make_pair(wl, path=M.PATH_STREAMING)
+    offsets = torch.tensor([0.0, -150.0, 150.0, -70.0, 70.0, -110.0, 110.0, 20.0], device=dev)
+    counts = {}
+    try:
+        for t in range(3):
+            arm = orc.select()
+            rd = gen.gathered_round(t, arm)
+            draft = (rd["draft"].float() + offsets.view(-1, 1, 1)).to(rd["draft"].dtype)
+            res = gpu.verify(rd["target"], draft, rd["tokens"], T, 31, want_diag=True)
+            out = orc.verify(rd["target"], draft, rd["tokens"].cpu().numpy(), T, 31)
+            compare_round(res, out, rd["target"], draft, T, 1.0, counts)
+            assert gpu.last_status() == 0
+    finally:
+        gpu.close()
+
+
 @pytest.mark.parametrize("path", PATHS)
 def test_defined_outcomes_of_anomalous_inputs(path):
     """NaN rows, masked (-inf) logits, out-of-range tokens: same defined outputs and status bits."""
