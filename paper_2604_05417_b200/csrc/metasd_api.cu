@@ -244,6 +244,10 @@ int metasd_verify(metasd_ctx *ctx, int32_t batch, int32_t k, const void *target_
     p.accepted_len = accepted_len; p.next_token = next_token; p.reward = reward; p.diag = diag;
     p.st = ctx->st; p.stats = ctx->stats; p.status = ctx->status;
     p.keep_permille = ctx->keep_permille;
+    {
+        const long long nvec = (long long)cfg.vocab * (long long)logit_size(cfg.logit_dtype) / 16;
+        p.keep_from_vec = (int32_t)(nvec - nvec * ctx->keep_permille / 1000);
+    }
     p.k1_stages = ctx->k1_stages;
     p.grp_size = ctx->grp_size; p.grp_ctas = ctx->grp_ctas;
     p.grp_rec = ctx->grp_rec; p.grp_min = ctx->grp_min; p.grp_count = ctx->grp_count;

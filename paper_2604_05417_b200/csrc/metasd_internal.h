@@ -64,6 +64,7 @@ struct VerifyParams {
     uint32_t *status;
     int32_t vector_ok; // rows are 16-byte aligned and a whole number of 16-byte vectors
     int32_t keep_permille;   // share of every row (its end) that the first sweep asks L2 to keep
+    int32_t keep_from_vec;   // the same as an index: first 16-byte vector of a row in the kept share
     int32_t k1_stages;       // depth of the row-statistics kernel's cp.async pipeline (0 or 1: plain loads)
     // split streaming path: grp_size CTAs share a row pair (0: one CTA per row pair)
     int32_t grp_size;

@@ -52,7 +52,7 @@ __global__ void __launch_bounds__(K1_THREADS) row_stats_kernel(const VerifyParam
     MaxSum sa = {METASD_NEG_BIG, 0.f}, sb = {METASD_NEG_BIG, 0.f};
     ArgMax am = {METASD_NEG_BIG, 0x7FFFFFFF};
     const uint64_t keep = l2_policy_evict_last(), drop = l2_policy_evict_first();
-    const int keep_from = nvec - (int)((long long)nvec * p.keep_permille / 1000);
+    const int keep_from = p.keep_from_vec;   // first 16-byte vector of a row that L2 is asked to keep (set by the host)
     for (int i = tid; i < nvec; i += K1_THREADS) {
         float xa[VEC], xb[VEC];
         if constexpr (VECTOR) {
@@ -213,7 +213,7 @@ __global__ void __launch_bounds__(THREADS, MINB) row_stats_staged_kernel(const V
     MaxSum sa = {METASD_NEG_BIG, 0.f}, sb = {METASD_NEG_BIG, 0.f};
     ArgMax am = {METASD_NEG_BIG, 0x7FFFFFFF};
     const uint64_t keep = l2_policy_evict_last(), drop = l2_policy_evict_first();
-    const int keep_from = nvec - (int)((long long)nvec * p.keep_permille / 1000);
+    const int keep_from = p.keep_from_vec;   // first 16-byte vector of a row that L2 is asked to keep (set by the host)
     auto request1 = [&](int n) {   // one group per call, empty past the end: the group count stays in step
         if (n < n_trip) {
             const int i = tid + n * THREADS;
