@@ -184,7 +184,7 @@ __device__ __forceinline__ uint4 lds16(uint32_t addr)
     return v;
 }
 
-template <typename LT, int D, int THREADS, int MINB>
+template <typename LT, int D, int THREADS, int MINB, bool BONUS_LAST>
 __global__ void __launch_bounds__(THREADS, MINB) row_stats_staged_kernel(const VerifyParams p)
 {
     static_assert(D >= 2, "at least two stages");
@@ -192,12 +192,19 @@ __global__ void __launch_bounds__(THREADS, MINB) row_stats_staged_kernel(const V
     constexpr int NWARP = THREADS / 32;
     constexpr uint32_t ROW_STRIDE = THREADS * 16, STAGE_STRIDE = 2 * ROW_STRIDE;
     extern __shared__ __align__(16) unsigned char stage_mem[];   // [D][2 rows][THREADS] 16-byte slots
-    const int j = blockIdx.x, b = blockIdx.y;
+    // Blocks are dispatched in index order.  BONUS_LAST: the row pairs come first and the bonus rows (one row, half
+    // the work) last, so that the launch ends on its shortest items (measured: better for the bf16 geometry, worse
+    // for the fp32 one, which keeps the bonus rows interleaved).
+    const int first_bonus = BONUS_LAST ? p.batch * p.k : 0x7FFFFFFF;
+    const int b = BONUS_LAST ? ((int)blockIdx.x < first_bonus ? (int)blockIdx.x / p.k : (int)blockIdx.x - first_bonus)
+                             : (int)blockIdx.x / (p.k + 1);
+    const int kb = drafted(p.draft_len, b, p.k);
+    const int j = BONUS_LAST ? ((int)blockIdx.x < first_bonus ? (int)blockIdx.x - b * p.k : kb)
+                             : (int)blockIdx.x - b * (p.k + 1);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const float c = p.c;
-    const int kb = drafted(p.draft_len, b, p.k);
-    if (j > kb) return;   // behind this sequence's bonus row: nothing to read
-    const bool pair = j < kb;
+    if (j > kb || (BONUS_LAST && (int)blockIdx.x < first_bonus && j == kb)) return;   // behind the bonus row, or the bonus row's
+    const bool pair = j < kb;                                           // own block does it
 
     const uint4 *a4 = reinterpret_cast<const uint4 *>(reinterpret_cast<const LT *>(p.target) + ((size_t)b * (p.k + 1) + j) * p.V);
     const uint4 *d4 = pair ? reinterpret_cast<const uint4 *>(draft_rows<LT>(p, b) + ((size_t)b * p.k + j) * p.V) : nullptr;
@@ -368,13 +375,13 @@ __global__ void __launch_bounds__(THREADS, MINB) row_stats_staged_kernel(const V
     }
 }
 
-template <typename LT, int D, int THREADS, int MINB>
+template <typename LT, int D, int THREADS, int MINB, bool BONUS_LAST>
 static cudaError_t launch_staged(const VerifyParams &p, dim3 grid, cudaStream_t stream)
 {
     const size_t smem = (size_t)D * 2 * THREADS * 16;
-    cudaError_t e = cudaFuncSetAttribute(row_stats_staged_kernel<LT, D, THREADS, MINB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(row_stats_staged_kernel<LT, D, THREADS, MINB, BONUS_LAST>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    row_stats_staged_kernel<LT, D, THREADS, MINB><<<grid, THREADS, smem, stream>>>(p);
+    row_stats_staged_kernel<LT, D, THREADS, MINB, BONUS_LAST><<<grid, THREADS, smem, stream>>>(p);
     return cudaSuccess;
 }
 
@@ -972,8 +979,9 @@ static cudaError_t launch_streaming_t(const VerifyParams &p, cudaStream_t stream
         // many small CTAs (4 x 384 threads per SM); fp32 rows (4 logits per 16 bytes) are bound by memory and want
         // few row pairs in flight and a large share of each kept in shared memory (1 x 1024 threads per SM).
         cudaError_t e;
-        if constexpr (sizeof(LT) == 2) e = launch_staged<LT, 4, 384, 4>(p, g1, stream);
-        else e = launch_staged<LT, 4, 1024, 1>(p, g1, stream);
+        const dim3 gp((unsigned)p.batch * (unsigned)(p.k + 1));
+        if constexpr (sizeof(LT) == 2) e = launch_staged<LT, 4, 384, 4, true>(p, gp, stream);
+        else e = launch_staged<LT, 4, 1024, 1, false>(p, gp, stream);
         if (e != cudaSuccess) return e;
     } else if (p.vector_ok) {
         row_stats_kernel<LT, true><<<g1, K1_THREADS, 0, stream>>>(p);
