@@ -221,23 +221,21 @@ __global__ void __launch_bounds__(THREADS, MINB) row_stats_staged_kernel(const V
     ArgMax am = {METASD_NEG_BIG, 0x7FFFFFFF};
     const uint64_t keep = l2_policy_evict_last(), drop = l2_policy_evict_first();
     const int keep_from = p.keep_from_vec;   // first 16-byte vector of a row that L2 is asked to keep (set by the host)
-    auto request1 = [&](int n) {   // one group per call, empty past the end: the group count stays in step
-        if (n < n_trip) {
-            const int i = tid + n * THREADS;
-            const uint64_t pol = i >= keep_from ? keep : drop;
-            const uint32_t dst = slot0 + (uint32_t)(n % D) * STAGE_STRIDE;
+    // One group of copies per call, empty past the end: the group count stays in step with the trips.
+    auto request1 = [&](int m, int slot, uint64_t pol) {
+        if (m < n_trip) {
+            const int i = tid + m * THREADS;
+            const uint32_t dst = slot0 + (uint32_t)slot * STAGE_STRIDE;
             cp_async16(dst, a4 + i, pol);
             if (pair) cp_async16(dst + ROW_STRIDE, d4 + i, pol);
         }
         cp_async_commit();
     };
-#pragma unroll
-    for (int n = 0; n < D - 1; ++n) request1(n);
-#pragma unroll 4
-    for (int n = 0; n < n_trip; ++n) {
-        request1(n + D - 1);
+    // Trip n of sweep 1 (its vectors sit in slot n mod D): first ask for the trip D - 1 ahead.
+    auto trip1 = [&](int n, int slot, uint64_t pol) {
+        request1(n + D - 1, (slot + D - 1) % D, pol);
         cp_async_wait<D - 1>();   // all but the D - 1 youngest groups have landed: trip n's is among them
-        const uint32_t src = slot0 + (uint32_t)(n % D) * STAGE_STRIDE;
+        const uint32_t src = slot0 + (uint32_t)slot * STAGE_STRIDE;
         const int i = tid + n * THREADS;
         float xa[VEC];
         Logit<LT>::unpack(lds16(src), xa);
@@ -265,7 +263,28 @@ __global__ void __launch_bounds__(THREADS, MINB) row_stats_staged_kernel(const V
 #pragma unroll
             for (int e = 0; e < VEC; ++e) sb.s += ex2(fmaf(xb[e], c, nma));
         }
+    };
+    // The trips run in groups of D so that the slot of every copy and read is a constant, and in two phases so that
+    // the L2 policy is one too: requests below the kept share of the row ask L2 to drop the line, the rest to keep it
+    // (the boundary is rounded down to a whole group: a few vectors more are kept).
+    const int m_keep = keep_from > tid ? (keep_from - tid + THREADS - 1) / THREADS : 0;   // first request that is kept
+    const int groups = n_trip / D;
+    int groups_drop = (m_keep - (D - 1)) / D;
+    groups_drop = groups_drop < 0 ? 0 : (groups_drop > groups ? groups : groups_drop);
+#pragma unroll
+    for (int m = 0; m < D - 1; ++m) request1(m, m, m >= m_keep ? keep : drop);
+    int n = 0;
+    for (int g = 0; g < groups_drop; ++g, n += D) {
+#pragma unroll
+        for (int u = 0; u < D; ++u) trip1(n + u, u, drop);
     }
+    for (int g = groups_drop; g < groups; ++g, n += D) {
+#pragma unroll
+        for (int u = 0; u < D; ++u) trip1(n + u, u, keep);
+    }
+#pragma unroll
+    for (int u = 0; u < D - 1; ++u)
+        if (n + u < n_trip) trip1(n + u, u, keep);
     cp_async_wait<0>();
     sb.m = sa.m;   // the draft row's sum is relative to the target row's maximum
 
@@ -333,12 +352,12 @@ __global__ void __launch_bounds__(THREADS, MINB) row_stats_staged_kernel(const V
     if (pair) {
         const float nma = sh_bcast[4], nmb = sh_bcast[5], ia = sh_bcast[6];
         float acc = 0.f;
-#pragma unroll 4
-        for (int n = n_trip - 1; n >= 0; --n) {
+        // Trip n of sweep 2 from its slot; the slot is then refilled with the trip D further down.
+        auto trip2 = [&](int n, int slot) {
             // the first D trips are still in their slots from sweep 1; the group of a later one was committed D trips
             // ago, so at most D - 1 younger groups may still be pending
             cp_async_wait<D - 1>();
-            const uint32_t src = slot0 + (uint32_t)(n % D) * STAGE_STRIDE;
+            const uint32_t src = slot0 + (uint32_t)slot * STAGE_STRIDE;
             float xa[VEC], xb[VEC];
             Logit<LT>::unpack(lds16(src), xa);
             Logit<LT>::unpack(lds16(src + ROW_STRIDE), xb);
@@ -351,6 +370,17 @@ __global__ void __launch_bounds__(THREADS, MINB) row_stats_staged_kernel(const V
                 cp_async16(src + ROW_STRIDE, d4 + i, drop);
             }
             cp_async_commit();
+        };
+        // the ragged top first, then whole groups downwards with constant slots
+        int n = n_trip - 1;
+        for (; n >= 0 && (n + 1) % D != 0; --n) trip2(n, n % D);
+        for (; n >= D; n -= D) {   // n + 1 is a multiple of D and a whole group lies below: every refill is real
+#pragma unroll
+            for (int u = 0; u < D; ++u) trip2(n - u, D - 1 - u);
+        }
+        if (n >= 0) {
+#pragma unroll
+            for (int u = 0; u < D; ++u) trip2(n - u, D - 1 - u);
         }
         cp_async_wait<0>();
         double w = warp_sum((double)(acc * ia));
