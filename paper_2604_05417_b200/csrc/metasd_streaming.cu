@@ -1005,12 +1005,13 @@ static cudaError_t launch_streaming_t(const VerifyParams &p, cudaStream_t stream
                                         dim3(KS_THREADS), args, 0, stream);
         if (e != cudaSuccess) return e;
     } else if (p.vector_ok && p.k1_stages > 1) {
-        // Measured on B200: bf16 rows (8 logits per 16 bytes) are bound by arithmetic as much as by memory and want
-        // many small CTAs (4 x 384 threads per SM); fp32 rows (4 logits per 16 bytes) are bound by memory and want
-        // few row pairs in flight and a large share of each kept in shared memory (1 x 1024 threads per SM).
+        // Measured on B200: bf16 rows (8 logits per 16 bytes) are bound by arithmetic as much as by memory: 3 x 512
+        // threads per SM (4 x 384 is as fast in short runs but moves 7 % more HBM bytes, which costs clock under
+        // the power cap); fp32 rows (4 logits per 16 bytes) are bound by memory and want few row pairs in flight
+        // and a large share of each kept in shared memory: 1 x 1024 threads per SM.
         cudaError_t e;
         const dim3 gp((unsigned)p.batch * (unsigned)(p.k + 1));
-        if constexpr (sizeof(LT) == 2) e = launch_staged<LT, 4, 384, 4, true>(p, gp, stream);
+        if constexpr (sizeof(LT) == 2) e = launch_staged<LT, 4, 512, 3, true>(p, gp, stream);
         else e = launch_staged<LT, 4, 1024, 1, false>(p, gp, stream);
         if (e != cudaSuccess) return e;
     } else if (p.vector_ok) {
