@@ -1008,11 +1008,11 @@ static cudaError_t launch_streaming_t(const VerifyParams &p, cudaStream_t stream
         // Measured on B200: bf16 rows (8 logits per 16 bytes) are bound by arithmetic as much as by memory: 3 x 512
         // threads per SM (4 x 384 is as fast in short runs but moves 7 % more HBM bytes, which costs clock under
         // the power cap); fp32 rows (4 logits per 16 bytes) are bound by memory and want few row pairs in flight
-        // and a large share of each kept in shared memory: 1 x 1024 threads per SM.
+        // and a large share of each kept in shared memory: 1 x 1024 threads per SM, 6 stages (192 KB).
         cudaError_t e;
         const dim3 gp((unsigned)p.batch * (unsigned)(p.k + 1));
         if constexpr (sizeof(LT) == 2) e = launch_staged<LT, 4, 512, 3, true>(p, gp, stream);
-        else e = launch_staged<LT, 4, 1024, 1, false>(p, gp, stream);
+        else e = launch_staged<LT, 6, 1024, 1, false>(p, gp, stream);
         if (e != cudaSuccess) return e;
     } else if (p.vector_ok) {
         row_stats_kernel<LT, true><<<g1, K1_THREADS, 0, stream>>>(p);
