@@ -65,9 +65,9 @@ def measured_peak_gbs():
 # DRAM bytes (read + write) of ONE launch of the dominant kernel, from the one-pass ncu capture of the full-size
 # launch that profiles/row_stats_staged_kernel.md summarises.  An entry is removed when its kernel changes.
 KNOWN_TRAFFIC = {
-    ("cfg4_greedy", "streaming"): 3.600e9 + 3.3e6,
-    ("cfg5_fp32_stress", "streaming"): 6.979e9 + 3.7e6,
-    ("cfg3_tasks", "streaming"): 1.333e9 + 3.3e6,
+    ("cfg4_greedy", "streaming"): 3.386e9 + 3.4e6,
+    ("cfg5_fp32_stress", "streaming"): 6.948e9 + 3.4e6,
+    ("cfg3_tasks", "streaming"): 1.238e9 + 5.9e6,
 }
 
 
