@@ -5,7 +5,7 @@ Comparison rules (what "results identical to the oracle" means here):
   * p_x, q_x, d_TV per position and the reward: within 1e-5 absolute;
   * accept bits: identical, except where the uniform lies within 1e-6 of p(x)/q(x) (counted);
   * sampled next_token: identical, except where the oracle's CDF margin is below 1e-6 and the GPU
-    token is the neighbouring token with mass (counted);
+    token is its neighbour in the CDF: the tokens strictly between them carry at most 2e-6 of the mass (counted);
   * arm choices: identical; a difference is tolerated only when the oracle's index gap is below 1e-6
     (counted, then the GPU state is re-synchronised from the oracle's).
 """
@@ -109,10 +109,13 @@ def compare_round(res, out, target, draft, T, reward_T, counts):
             assert out["sample_margin"][b] < NEAR, "sampled token differs away from a CDF edge"
             j = int(out["accepted_len"][b])
             w = _row_weights(tgt[b, j], drf[b, j] if j < k else None, T)
-            mass = np.nonzero(w > 0)[0]
-            pos = int(np.searchsorted(mass, out["next_token"][b]))
-            neighbours = set(mass[max(0, pos - 1): pos + 2].tolist())
-            assert int(g_tok[b]) in neighbours, "GPU token is not the neighbouring token with mass"
+            # the two tokens must be neighbours in the CDF: what lies strictly between them carries (next to) no mass.
+            # In float64 that is "the neighbouring token with mass"; fp32 may flush weights of 1e-12 that float64
+            # still sees, so the bound is on the mass in between, not on the count of tokens.
+            lo, hi = sorted((int(g_tok[b]), int(out["next_token"][b])))
+            between = float(w[lo + 1:hi].sum())
+            assert 0 <= lo and hi < len(w) and between <= 2 * NEAR * float(w.sum()), \
+                "GPU token is not the oracle's neighbour in the CDF"
         counts["near_tie_token"] = counts.get("near_tie_token", 0) + int(tok_mism.sum())
     counts["rounds"] = counts.get("rounds", 0) + 1
     counts["tokens"] = counts.get("tokens", 0) + int((g_len + 1).sum())
