@@ -111,6 +111,17 @@ def test_pure_exploration_then_commit(path, N, budget):
     assert c["rounds"] == budget + 12 and c.get("near_tie_arm", 0) == 0
 
 
+@pytest.mark.parametrize("dtype,V,T,k,bandit", [("bf16", 152064, 1.0, 8, "ucb"), ("fp32", 128256, 1.0, 5, "ducb"),
+                                                ("bf16", 50264, 1.3, 6, "petc")])
+def test_many_rounds_on_large_vocabularies(dtype, V, T, k, bandit):
+    """Lock-step rounds at the benchmark's vocabulary sizes (several trips of every staging depth, ragged last trip),
+    sampled mode, pointer-table inputs: every round's outputs and the bandit state follow the oracle."""
+    from _harness import run_lockstep
+    wl = base(B=12, N=4, k=k, V=V, sigmas=(0.3, 1.0, 2.0, 3.0)).scaled(dtype=dtype, temperature=T, tau=20)
+    c = report(run_lockstep(wl, rounds=12, seed=V % 97, path=M.PATH_STREAMING, bandit=bandit, table_mode=True))
+    assert c["rounds"] == 12 and c["status"] == 0 and c["max_err_D"] < 5e-6
+
+
 @pytest.mark.parametrize("path", PATHS)
 def test_pointer_table_mode(path):
     """The kernel indexes a table of K drafter tensors and a [K,B,k] token table by arm."""
