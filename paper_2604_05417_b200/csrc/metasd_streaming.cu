@@ -219,7 +219,8 @@ __global__ void __launch_bounds__(THREADS, MINB) row_stats_staged_kernel(const V
     // after the sweep; if not, that row's statistics are redone relative to its own maximum.
     MaxSum sa = {METASD_NEG_BIG, 0.f}, sb = {METASD_NEG_BIG, 0.f};
     ArgMax am = {METASD_NEG_BIG, 0x7FFFFFFF};
-    const uint64_t keep = l2_policy_evict_last(), drop = l2_policy_evict_first();
+    // a bonus row is read once: nothing of it is worth keeping in L2
+    const uint64_t drop = l2_policy_evict_first(), keep = pair ? l2_policy_evict_last() : drop;
     const int keep_from = p.keep_from_vec;   // first 16-byte vector of a row that L2 is asked to keep (set by the host)
     // One group of copies per call, empty past the end: the group count stays in step with the trips.
     auto request1 = [&](int m, int slot, uint64_t pol) {
