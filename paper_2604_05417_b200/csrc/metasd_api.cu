@@ -123,7 +123,7 @@ int metasd_init(metasd_ctx **out, const metasd_config *cfg)
     c->cfg = *cfg;
     {   // the best measured values on B200 for 128k-152k vocabularies (METASD_KEEP_PERMILLE overrides, for tuning)
         const char *kp = getenv("METASD_KEEP_PERMILLE");
-        const int v = kp && *kp ? atoi(kp) : (cfg->logit_dtype == METASD_BF16 ? 750 : 800);
+        const int v = kp && *kp ? atoi(kp) : (cfg->logit_dtype == METASD_BF16 ? 750 : 900);
         c->keep_permille = v < 0 ? 0 : (v > 1000 ? 1000 : v);
     }
     {
