@@ -203,8 +203,9 @@ __global__ void __launch_bounds__(THREADS, MINB) row_stats_staged_kernel(const V
                              : (int)blockIdx.x - b * (p.k + 1);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const float c = p.c;
-    if (j > kb || (BONUS_LAST && (int)blockIdx.x < first_bonus && j == kb)) return;   // behind the bonus row, or the bonus row's
-    const bool pair = j < kb;                                           // own block does it
+    // nothing to do behind the sequence's bonus row; with BONUS_LAST the bonus row belongs to its own late block
+    if (j > kb || (BONUS_LAST && (int)blockIdx.x < first_bonus && j == kb)) return;
+    const bool pair = j < kb;
 
     const uint4 *a4 = reinterpret_cast<const uint4 *>(reinterpret_cast<const LT *>(p.target) + ((size_t)b * (p.k + 1) + j) * p.V);
     const uint4 *d4 = pair ? reinterpret_cast<const uint4 *>(draft_rows<LT>(p, b) + ((size_t)b * p.k + j) * p.V) : nullptr;
