@@ -256,6 +256,9 @@ def main():
                 "traffic": known_traffic(wl.name, path_name) if not (args.batch or args.k or args.ragged) else None, "peak_kind": "of " + peak_kind,
                 "algorithmic_bytes_per_launch": bytes_round, "kernel_ms": kernel_ms,
                 "frac_of_8TBs_nominal": achieved / 8000.0,
+                # the same over the first timed steps only: before the power cap pulls the SM clock down
+                "first_40_steps": {"kernel_ms": statistics.mean(step_ms[:40]),
+                                   "frac": bytes_round / (statistics.mean(step_ms[:40]) * 1e-3) / 1e9 / peak},
                 "note": "duration = CUDA events around select+verify of one step (%s path)" % path_name}
 
     result = {
