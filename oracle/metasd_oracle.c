@@ -5,8 +5,10 @@
  * speculative-sampling verification (Algorithm 4, the verification loop and the
  * bonus token), the block-divergence reward (Definition 2 / Eq. 4) and the
  * block-efficiency reward (Sec. 2.3), and the bandit policies MetaSD-UCB
- * (Algorithm 2), Discounted UCB (Appendix, "Discounted UCB in MetaSD") and
- * Sliding-window UCB (Appendix, "Sliding-window UCB in MetaSD").
+ * (Algorithm 2), Discounted UCB (Appendix, "Discounted UCB in MetaSD"),
+ * Sliding-window UCB (Appendix, "Sliding-window UCB in MetaSD"), MetaSD-EXP3 and the
+ * uniformly random baseline, and Pure exploration-then-commit with Sequential Halving
+ * (the algorithm boxes of those names in the switching-cost appendix).
  *
  * Only tests, the smoke check and the benchmark's CPU-baseline leg may call this
  * file.  It shares no code with the CUDA path.  Everything is written in the
@@ -20,6 +22,11 @@
  *   D-UCB normaliser (discounted count) and SW-UCB empty-window rule:
  *   reductions to UCB pinned; the readings themselves ............. parity unpinned
  *   inverse-CDF tie rule (token-id order, strict >) ................ parity unpinned
+ *   EXP3 update, probabilities and draw; Rand ...................... pinned
+ *   EXP3 mixing parameter value; which Philox word draws the arm .. parity unpinned
+ *   Sequential Halving / PETC schedule, halving, error bound ....... pinned
+ *   order of pulls inside a halving phase .......................... parity unpinned
+ *   per-sequence draft lengths (reduction to the fixed length) ..... pinned
  */
 #include <math.h>
 #include <stdint.h>
