@@ -329,11 +329,12 @@ def test_petc_schedule_worked_by_hand_for_four_drafters():
 
 
 def test_petc_phase_sums_restart_and_only_the_current_phase_counts():
-    # drafter 3 is best in phase 0 and worst afterwards: with sums restarted it loses phase 1 to drafter 1
+    # drafter 3 wins phase 0 by far (2 x 1.0 against 2 x 0.55) and is slightly worse afterwards (4 x 0.5 against
+    # 4 x 0.55): with sums restarted it loses phase 1 to drafter 1; carried over (4.0 against 3.3) it would win
     def reward(a, t, g):
         if a == 3:
-            return 1.0 if t < 8 else 0.0
-        return [0.1, 0.6, 0.2][a]
+            return 1.0 if t < 8 else 0.5
+        return [0.1, 0.55, 0.2][a]
     arms, _, orc = run_bandit(O.PETC, 4, reward, 20, tau=16)
     assert sorted(set(arms[8:16].tolist())) == [1, 3]
     assert (arms[16:] == 1).all()
@@ -344,7 +345,7 @@ def test_petc_phase_sums_restart_and_only_the_current_phase_counts():
 def test_petc_halves_ceil_log2_times_and_spends_at_most_its_budget(K):
     budget = 12 * K
     L = math.ceil(math.log2(K)) if K > 1 else 0
-    rng_means = np.random.RandomState(K).rand(K)
+    rng_means = np.random.RandomState(K).permutation(np.linspace(0.1, 0.9, K)) if K > 1 else np.array([0.5])
     arms, _, orc = run_bandit(O.PETC, K, lambda a, t, g: rng_means[a] + 0.01 * g.rand(), budget + 25, tau=budget)
     # exploration length: sum over phases of n_r |S_r| with |S_{r+1}| = ceil(|S_r| / 2)
     size, spent, sizes = K, 0, []
@@ -363,6 +364,8 @@ def test_petc_halves_ceil_log2_times_and_spends_at_most_its_budget(K):
         block = arms[pos:pos + n * s]
         values, counts = np.unique(block, return_counts=True)
         assert len(values) == s and (counts == n).all()
+        # the means are far apart next to the noise: S_r is exactly the |S_r| best drafters
+        assert set(values.tolist()) == set(np.argsort(-rng_means)[:s].tolist())
         pos += n * s
     # with well separated means the best drafter survives
     assert tail[0] == int(np.argmax(rng_means))
