@@ -521,3 +521,71 @@ def test_ragged_round_equals_the_fixed_length_round_on_the_truncated_rows():
     plain = O.OracleMetaSD(cfg).verify(target, draft, tokens, 1.0, 77, update=False)
     for key in ("accepted_len", "next_token", "reward", "D", "accept"):
         assert np.array_equal(full[key], plain[key])
+
+
+# ------------------------------------------------------------------ random-number keying, pointer-table mode
+def _documented_uniforms(seed, sequence, round_, position):
+    """The convention fixed for both sides: Philox4x32-10 with key (seed low, seed high) at counter
+    (sequence, round, position, 0); word 0 is the accept test's uniform, word 1 the draw's; top 24 bits."""
+    w = O.philox4x32_10([sequence, round_, position, 0], [seed & 0xFFFFFFFF, seed >> 32])
+    return (int(w[0]) >> 8) / 2.0 ** 24, (int(w[1]) >> 8) / 2.0 ** 24
+
+
+def test_round_uniforms_follow_the_documented_counter_and_words():
+    for seed, seq, rnd, pos in [(0, 0, 0, 0), (7, 1, 2, 3), (0xDEADBEEF12345678, 4000000000, 17, 5),
+                                (1 << 40, 9, 300, 16), (555, 3, 1, 2), (555, 1, 3, 2), (555, 2, 1, 3)]:
+        assert O.round_uniforms(seed, seq, rnd, pos) == _documented_uniforms(seed, seq, rnd, pos)
+    # swapping any two counter fields gives other numbers (the three cases above with 1, 2, 3 permuted)
+    assert len({O.round_uniforms(555, *c) for c in [(3, 1, 2), (1, 3, 2), (2, 1, 3)]}) == 3
+
+
+def test_batch_round_draws_its_uniforms_by_sequence_round_and_position():
+    """The batch call, replayed sequence by sequence with uniforms rebuilt from the Philox block of
+    (sequence_base + b, round of b, position): accept uniforms from word 0, the draw at position j from word 1
+    of position j's block.  A swapped counter field or word would move tokens and accepted lengths."""
+    rng = np.random.RandomState(12)
+    B, k, V, base, seed = 24, 4, 61, 1000, 0x1234ABCD5678
+    target = (rng.randn(B, k + 1, V) * 2).astype(np.float32)
+    draft = (target[:, :k] + rng.randn(B, k, V)).astype(np.float32)
+    tokens = rng.randint(0, V, size=(B, k)).astype(np.int32)
+    orc = O.OracleMetaSD(O.OracleConfig(max_batch=B, n_drafters=3, vocab=V, sequence_base=base))
+    orc.t[:] = rng.randint(0, 50, size=B)
+    rounds = orc.t.copy()
+    out = orc.verify(target, draft, tokens, 0.9, seed, update=False)
+    lens = set()
+    for b in range(B):
+        ua = [_documented_uniforms(seed, base + b, int(rounds[b]), j)[0] for j in range(k)]
+        us = [_documented_uniforms(seed, base + b, int(rounds[b]), j)[1] for j in range(k + 1)]
+        assert np.array_equal(out["u_accept"][b], ua)
+        one = O.verify_sequence(target[b], draft[b], tokens[b], 0.9, ua, us)
+        assert one["accepted_len"] == out["accepted_len"][b] and one["next_token"] == out["next_token"][b]
+        assert np.array_equal(one["accept"], out["accept"][b])
+        lens.add(one["accepted_len"])
+    assert len(lens) >= 3          # rejections at several positions and full acceptance are all covered
+
+
+def test_pointer_table_mode_equals_gathered_mode():
+    """Reading drafter arm[b]'s rows through the table of K tensors is the same round as reading rows that
+    were gathered by arm beforehand: every output, bit for bit, and the same bandit state afterwards."""
+    rng = np.random.RandomState(3)
+    B, K, k, V = 7, 3, 3, 53
+    for bandit in (O.UCB, O.SWUCB):
+        tab = O.OracleMetaSD(O.OracleConfig(max_batch=B, n_drafters=K, vocab=V, bandit=bandit, tau=4))
+        gat = O.OracleMetaSD(O.OracleConfig(max_batch=B, n_drafters=K, vocab=V, bandit=bandit, tau=4))
+        for t in range(9):
+            target = (rng.randn(B, k + 1, V) * 2).astype(np.float32)
+            drafts = [(target[:, :k] + (0.3 + i) * rng.randn(B, k, V)).astype(np.float32) for i in range(K)]
+            tokens = rng.randint(0, V, size=(K, B, k)).astype(np.int32)
+            arm = gat.select()
+            assert np.array_equal(arm, tab.select())
+            rows = np.stack(drafts)[arm, np.arange(B)]
+            toks = tokens[arm, np.arange(B)]
+            # a table rotated by one drafter gives another round: the table really is indexed by the arm
+            wrong = tab.verify(target, None, toks, 1.0, 99, drafter_tables=[drafts[(i + 1) % K] for i in range(K)],
+                               update=False)
+            a = tab.verify(target, None, toks, 1.0, 99, drafter_tables=drafts)
+            b = gat.verify(target, rows, toks, 1.0, 99)
+            for key in ("accepted_len", "next_token", "reward", "p_x", "q_x", "D", "accept", "u_accept", "sample_margin"):
+                assert np.array_equal(a[key], b[key]), key
+            assert not (wrong["D"] == a["D"]).any()
+        assert np.array_equal(tab.stat_a, gat.stat_a) and np.array_equal(tab.t, gat.t)
