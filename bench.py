@@ -50,6 +50,15 @@ def parse_args():
     ap.add_argument("--k", type=int, default=0, help="override the workload's draft length (the N_max sweep)")
     ap.add_argument("--ragged", action="store_true",
                     help="per-sequence draft lengths, uniform in 1..k (seeded); bytes are counted per sequence")
+    ap.add_argument("--row-kernel", default="auto", choices=["auto", "plain", "staged", "bulk"])
+    ap.add_argument("--row-threads", type=int, default=0)
+    ap.add_argument("--row-stages", type=int, default=0)
+    ap.add_argument("--keep-permille", type=int, default=0)
+    ap.add_argument("--order", default="rank", choices=["rank", "reversed", "shuffled"],
+                    help="where the likely tokens sit in the vocabulary (the draw walks it in id order)")
+    ap.add_argument("--sustained-seconds", type=float, default=1.0,
+                    help="length of the extra back-to-back leg that is run when the timed region is under half a second")
+    ap.add_argument("--no-parity", action="store_true")
     return ap.parse_args()
 
 
@@ -62,17 +71,15 @@ def measured_peak_gbs():
         return 6650.0, "fallback"
 
 
-# DRAM bytes (read + write) of ONE launch of the dominant kernel, from the one-pass ncu capture of the full-size
-# launch that profiles/row_stats_staged_kernel.md summarises.  An entry is removed when its kernel changes.
-KNOWN_TRAFFIC = {
-    ("cfg4_greedy", "streaming"): 3.386e9 + 3.4e6,
-    ("cfg5_fp32_stress", "streaming"): 6.735e9 + 3.7e6,
-    ("cfg3_tasks", "streaming"): 1.238e9 + 5.9e6,
-}
-
-
-def known_traffic(workload: str, path_name: str):
-    return KNOWN_TRAFFIC.get((workload, path_name))
+def known_traffic(kernel_key: str, workload: str):
+    """DRAM bytes (read + write) of one launch of the dominant kernel from the committed ncu capture of exactly this
+    kernel variant on this workload, or None when there is no such capture (a changed kernel has a new key)."""
+    try:
+        with open(os.path.join(ROOT, "profiles", "dram_traffic.json")) as f:
+            table = json.load(f)
+        return table["captures"].get(kernel_key, {}).get(workload)
+    except Exception:
+        return None
 
 
 class ClockSampler:
@@ -87,7 +94,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "20"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except Exception:
             self.proc = None
             return
@@ -97,10 +104,9 @@ class ClockSampler:
         self.thread = threading.Thread(target=pump, daemon=True)
         self.thread.start()
 
-    def stop(self, t_begin=0.0, t_end=float("inf")):
-        """Median SM clock and the throttle reasons of the samples taken in [t_begin, t_end]."""
+    def stop(self):
         if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+            return
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
@@ -108,10 +114,21 @@ class ClockSampler:
             self.proc.kill()
         if self.thread is not None:
             self.thread.join(timeout=2)
+        self.proc = None
+
+    def window(self, t_begin, t_end):
+        """Median SM clock and the throttle reasons of the samples taken in [t_begin, t_end]; a region shorter than
+        the sampling period takes the samples on either side of it."""
+        if not self.rows:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         clocks, reasons, mx = [], set(), None
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         inside = [r for ts, r in self.rows if t_begin <= ts <= t_end]
-        for r in (inside or [r for _, r in self.rows[-3:]]):
+        if not inside:
+            before = [r for ts, r in self.rows if ts < t_begin][-1:]
+            after = [r for ts, r in self.rows if ts > t_end][:1]
+            inside = before + after
+        for r in inside:
             try:
                 clocks.append(float(r[0]))
                 mx = float(r[1])
@@ -135,22 +152,68 @@ def oracle_sample_run(wl, host_rounds, seconds: float):
         orc = O.OracleMetaSD(O.OracleConfig(max_batch=n_seq, n_drafters=wl.N, vocab=wl.V,
                                             bandit={"ucb": 0, "ducb": 1, "swucb": 2}[wl.bandit], beta=wl.beta,
                                             gamma=wl.gamma, tau=wl.tau))
-        tokens = 0
+        tokens, outs = 0, []
         t0 = time.perf_counter()
         for r in range(rounds):
             tg, dr, tk = host_rounds[r % len(host_rounds)]
             out = orc.verify(tg[:n_seq], dr[:n_seq], tk[:n_seq].numpy(), wl.temperature, LIB_SEED)
             tokens += int((out["accepted_len"] + 1).sum())
-        return tokens, time.perf_counter() - t0
+            outs.append(out)
+        return tokens, time.perf_counter() - t0, outs
 
     n0 = min(avail, cores)
-    _, dt = run(n0, 1)                                   # calibration (also warms the caches)
+    _, dt, _ = run(n0, 1)                                # calibration (also warms the caches)
     wall_per_round = max(dt, 1e-6) * (avail / n0)        # one round of all `avail` sequences
     n_seq = avail
     rounds = int(max(2, min(200, seconds / wall_per_round)))
-    tokens, dt = run(n_seq, rounds)
+    tokens, dt, outs = run(n_seq, rounds)
     return {"value": tokens / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": "%d sequences x %d rounds of %s (float64, OpenMP over sequences), %.1f s" % (n_seq, rounds, wl.name, dt)}
+            "sample": "%d sequences x %d rounds of %s (float64, OpenMP over sequences), %.1f s" % (n_seq, rounds, wl.name, dt)}, outs
+
+
+def parity_against_oracle(wl, M, host_rounds, outs, dev, tuning):
+    """The library on the very rounds the CPU-baseline leg gave the oracle (outside every timed region): what differs,
+    counted by the comparison rules of the parity tests.  Integers must agree except at the oracle's own near ties
+    (uniform within 1e-6 of p/q; CDF margin below 1e-6; index gap below 1e-6), floats within 1e-5."""
+    import numpy as np
+    n = outs[0]["accepted_len"].shape[0]
+    gpu = M.MetaSD(n, wl.N, wl.k, wl.V, dtype=wl.dtype, bandit=wl.bandit, beta=wl.beta, gamma=wl.gamma, window=wl.tau,
+                   device=dev.index, **tuning)
+    dev_rounds = [tuple(x[:n].to(dev) for x in hr) for hr in host_rounds]
+    rep = {"sequences": n, "rounds": len(outs), "near_tie_accept": 0, "near_tie_token": 0, "near_tie_arm": 0,
+           "mismatch_accept": 0, "mismatch_token": 0, "mismatch_arm": 0, "max_err_D": 0.0, "max_err_p": 0.0,
+           "max_err_reward": 0.0, "uniforms_identical": True}
+    greedy = not (wl.temperature > 0)
+    for r, out in enumerate(outs):
+        tg, dr, tk = dev_rounds[r % len(dev_rounds)]
+        arm_g = gpu.select().cpu().numpy()
+        differs = arm_g != out["arm"]
+        # a stored gap belongs to the selection that FOLLOWED the previous round
+        near = differs & (outs[r - 1]["next_gap"] < 1e-6) if r else np.zeros(n, dtype=bool)
+        rep["near_tie_arm"] += int(near.sum())
+        rep["mismatch_arm"] += int((differs & ~near).sum())
+        res = gpu.verify(tg, dr, tk, wl.temperature, LIB_SEED, want_diag=True)
+        p_x, q_x, D, u, acc = [x.cpu().numpy() for x in res.diag_fields()]
+        rep["uniforms_identical"] &= bool(np.array_equal(u.astype(np.float64), out["u_accept"]))
+        rep["max_err_D"] = max(rep["max_err_D"], float(np.abs(D - out["D"]).max()))
+        rep["max_err_p"] = max(rep["max_err_p"], float(np.abs(p_x - out["p_x"]).max()), float(np.abs(q_x - out["q_x"]).max()))
+        rep["max_err_reward"] = max(rep["max_err_reward"], float(np.abs(res.reward.cpu().numpy() - out["reward"]).max()))
+        bits = acc != out["accept"]
+        with np.errstate(divide="ignore", invalid="ignore"):
+            tie = np.abs(out["u_accept"] - out["p_x"] / out["q_x"]) < 1e-6
+        rep["near_tie_accept"] += int((bits & tie).sum())
+        rep["mismatch_accept"] += int((bits & ~tie).sum())
+        same_len = res.accepted_len.cpu().numpy() == out["accepted_len"]
+        rep["mismatch_accept"] += int((~same_len & ~bits.any(axis=1)).sum())
+        tok = (res.next_token.cpu().numpy() != out["next_token"]) & same_len
+        edge = tok & (out["sample_margin"] < 1e-6) & (not greedy)
+        rep["near_tie_token"] += int(edge.sum())
+        rep["mismatch_token"] += int((tok & ~edge).sum())
+    rep["status"] = gpu.last_status()
+    gpu.close()
+    rep["ok"] = bool(rep["mismatch_accept"] == 0 and rep["mismatch_token"] == 0 and rep["mismatch_arm"] == 0 and
+                     rep["uniforms_identical"] and max(rep["max_err_D"], rep["max_err_p"], rep["max_err_reward"]) < 1e-5)
+    return rep
 
 
 def main():
@@ -163,6 +226,8 @@ def main():
         wl = wl.scaled(B=args.batch)
     if args.k:
         wl = wl.scaled(k=args.k)
+    if args.order != "rank":
+        wl = wl.scaled(order=args.order)
 
     if args.impl == "reference":
         return reference_arm(args, wl, rank)
@@ -177,9 +242,15 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
 
     path = {"auto": M.PATH_AUTO, "streaming": M.PATH_STREAMING, "fused": M.PATH_FUSED}[args.path]
+    tuning = dict(row_kernel={"auto": M.ROWS_AUTO, "plain": M.ROWS_PLAIN, "staged": M.ROWS_STAGED, "bulk": M.ROWS_BULK}[args.row_kernel],
+                  row_threads=args.row_threads, row_stages=args.row_stages, keep_permille=args.keep_permille)
     msd = M.MetaSD(wl.B, wl.N, wl.k, wl.V, dtype=wl.dtype, bandit=wl.bandit, beta=wl.beta, gamma=wl.gamma,
-                   window=wl.tau, device=local_rank, path=path, sequence_base=rank * wl.B)
+                   window=wl.tau, device=local_rank, path=path, sequence_base=rank * wl.B, **tuning)
     path_name = {M.PATH_STREAMING: "streaming", M.PATH_FUSED: "fused"}[msd.resolved_path(wl.k)]
+    row_kernel = {M.ROWS_PLAIN: "plain", M.ROWS_STAGED: "staged", M.ROWS_BULK: "bulk"}[msd.resolved_row_kernel()]
+    # names the dominant kernel's variant: a capture of DRAM traffic counts only for the variant it was taken on
+    kernel_key = path_name if path_name == "fused" else "%s/%s/t%d/s%d/keep%d" % (
+        row_kernel, wl.dtype, args.row_threads, args.row_stages, args.keep_permille)
 
     # ---- inputs: R distinct rounds, every drafter's logits and tokens resident in HBM
     gen = RoundGenerator(wl, device=dev, seed=1000 + rank)
@@ -231,8 +302,27 @@ def main():
         ev[i][1].record()
     t_end.record()
     barrier()
-    clocks = sampler.stop(host_begin, time.time())
+    host_end = time.time()
     launches = msd.kernel_launches() - launches0
+    # ---- a timed region under half a second says little about sustained rounds (the power cap acts after a few
+    # hundred milliseconds): run an extra leg of back-to-back rounds and report it beside the timed one
+    sustained = None
+    if t_start.elapsed_time(t_end) < 500.0 and args.sustained_seconds > 0:
+        per_step = max(t_start.elapsed_time(t_end) / args.steps, 1e-3)
+        n_sus = int(min(20000, max(args.steps, args.sustained_seconds * 1e3 / per_step)))
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        sus_begin = time.time()
+        s0.record()
+        for i in range(n_sus):
+            step(i % n_all)
+        s1.record()
+        barrier()
+        sus_end = time.time()
+        sustained = {"steps": n_sus, "kernel_ms": s0.elapsed_time(s1) / n_sus, "window": (sus_begin, sus_end)}
+    time.sleep(0.05)
+    sampler.stop()
+    clocks = sampler.window(host_begin, host_end)
     total_ms = t_start.elapsed_time(t_end)
     step_ms = [a.elapsed_time(b) for a, b in ev]
     tokens = int(acc_all[args.warmup:].sum().item()) + args.steps * wl.B   # verified tokens: sum(N_acc + 1)
@@ -253,20 +343,26 @@ def main():
     peak, peak_kind = measured_peak_gbs()
     achieved = bytes_round / (kernel_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": known_traffic(wl.name, path_name) if not (args.batch or args.k or args.ragged) else None, "peak_kind": "of " + peak_kind,
+                "traffic": known_traffic(kernel_key, wl.name) if not (args.batch or args.k or args.ragged) else None,
+                "traffic_key": kernel_key, "peak_kind": "of " + peak_kind,
                 "algorithmic_bytes_per_launch": bytes_round, "kernel_ms": kernel_ms,
                 "frac_of_8TBs_nominal": achieved / 8000.0,
                 # the same over the first timed steps only: before the power cap pulls the SM clock down
                 "first_40_steps": {"kernel_ms": statistics.mean(step_ms[:40]),
                                    "frac": bytes_round / (statistics.mean(step_ms[:40]) * 1e-3) / 1e9 / peak},
-                "note": "duration = CUDA events around select+verify of one step (%s path)" % path_name}
+                "note": "duration = CUDA events around select+verify of one step (%s path, %s row kernel)" % (path_name, row_kernel)}
+    if sustained is not None:
+        ms = sustained["kernel_ms"]
+        roofline["sustained"] = {"steps": sustained["steps"], "kernel_ms": ms, "frac": bytes_round / (ms * 1e-3) / 1e9 / peak,
+                                 "clocks": sampler.window(*sustained["window"])}
 
     result = {
         "metric": METRIC, "value": tokens / (total_ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": wl.name, "B_per_gpu": wl.B, "N": wl.N, "k": wl.k, "V": wl.V, "logits": wl.dtype,
-                   "temperature": wl.temperature, "bandit": wl.bandit, "path": path_name,
+                   "temperature": wl.temperature, "bandit": wl.bandit, "path": path_name, "row_kernel": row_kernel,
+                   "vocab_order": wl.order,
                    "draft_len": "uniform 1..k per sequence" if args.ragged else "k for every sequence",
                    "l2": "inputs larger than L2: %.2f GB read per step, %d rotating input sets" % (bytes_round / 1e9, len(rounds))},
         "rounds_per_s": world * args.steps / (total_ms * 1e-3),
@@ -287,7 +383,9 @@ def main():
             draft = torch.stack([d[:n] for d in rd["drafts"]])[idx, torch.arange(n, device=dev)]
             toks = rd["tokens"][:, :n][idx, torch.arange(n, device=dev)]
             host.append((rd["target"][:n].cpu(), draft.cpu(), toks.cpu()))
-        result["cpu_baseline"] = oracle_sample_run(wl, host, args.cpu_seconds)
+        result["cpu_baseline"], outs = oracle_sample_run(wl, host, args.cpu_seconds)
+        if not args.no_parity:
+            result["parity"] = parity_against_oracle(wl, M, host, outs, dev, tuning)
     msd.close()
     if rank == 0:
         print(json.dumps(result))

@@ -1,8 +1,8 @@
 /*
  * metasd.h -- C ABI of the MetaSD draft-verify hot path on NVIDIA B200 (sm_100a).
  *
- * One MetaSD round (Algorithm 1 of the paper: "meta-draft a drafter following the bandit ->
- * one speculative-decoding step -> block-divergence reward -> update the bandit") for a batch of
+ * One MetaSD round (Algorithm 1 of the paper: the bandit picks a drafter, one speculative-decoding
+ * step runs with it, the alignment reward of that step updates the bandit) for a batch of
  * B independent sequences, each with its own bandit instance over K drafters:
  *
  *   metasd_select  : the drafter each sequence plays this round           (Algorithm 2, selection rule)
@@ -20,6 +20,9 @@
  *     state and its scratch; nothing is allocated after metasd_init.
  *   - Calls are asynchronous on the CUDA stream passed as `stream` (a cudaStream_t, typed void*
  *     so that this header needs no CUDA include); calls on one context must be stream-ordered.
+ *   - A context belongs to the device named in its configuration.  Every call that takes a context
+ *     makes that device current for its own duration and restores the caller's current device before
+ *     it returns; `stream` must be a stream of the context's device (or NULL).
  *   - Every function returns 0 (METASD_OK) or a negative metasd_error.  Device-side anomalies
  *     never trap: they set bits in the context's status word and produce the defined outputs
  *     described at metasd_last_status.
@@ -62,6 +65,16 @@ enum metasd_bandit {
 };
 enum metasd_reward { METASD_REWARD_BD = 0, METASD_REWARD_BE = 1 };
 
+/* How the row-statistics kernel of the streaming path brings logit rows on chip (16-byte aligned rows; rows
+ * that are not take plain scalar loads whatever is asked for). */
+enum metasd_row_kernel {
+    METASD_ROWS_AUTO = 0,    /* the fastest measured variant for the dtype */
+    METASD_ROWS_PLAIN = 1,   /* ld.global straight into registers */
+    METASD_ROWS_STAGED = 2,  /* per-thread cp.async into shared-memory slots, several trips ahead */
+    METASD_ROWS_BULK = 3     /* a persistent CTA per SM: one warp issues TMA bulk copies (cp.async.bulk, mbarrier
+                                completion) into a shared-memory ring, the other warps consume it */
+};
+
 /* Which kernels metasd_verify launches. */
 enum metasd_path {
     METASD_PATH_AUTO = 0,      /* the fastest measured path for the shape (currently: streaming) */
@@ -75,7 +88,8 @@ enum metasd_path {
 #define METASD_STATUS_NONFINITE 1u /* a row held NaN / +Inf or no finite entry */
 #define METASD_STATUS_TOKEN_OOR 2u /* a drafted token id was outside [0, V) */
 #define METASD_STATUS_Q_ZERO    4u /* the drafter gave probability 0 to its own drafted token */
-#define METASD_STATUS_TIMEOUT   8u /* a bounded wait on an asynchronous copy ran out: outputs of that call are undefined */
+#define METASD_STATUS_TIMEOUT   8u /* a bounded device-side wait on an asynchronous copy ran out (see wait_poll_limit): the
+                                      call still ends, its outputs are undefined, the context stays usable */
 #define METASD_STATUS_BAD_LENGTH 32u /* a registered per-sequence draft length was outside 1 .. k: it was clamped */
 #define METASD_STATUS_BAD_POINTER 16u /* the drafter table of a call held a NULL or misaligned entry: its rows are never
                                         read and the outputs of the sequences that played that drafter are meaningless */
@@ -104,6 +118,17 @@ typedef struct metasd_config {
     double beta;
     double gamma;
     double reward_temperature;  /* softmax temperature of the reward when verifying greedily */
+    /* Tuning and test fields; 0 everywhere (what metasd_default_config writes) selects the measured defaults. */
+    int32_t row_kernel;         /* metasd_row_kernel */
+    int32_t row_threads;        /* threads per CTA of the row-statistics kernel; only the built shapes are accepted */
+    int32_t row_stages;         /* depth of its shared-memory staging; only the built shapes are accepted */
+    int32_t keep_permille;      /* share (its end, in 1/1000) of every row that the first sweep asks L2 to keep for the
+                                   second; 0 = default, negative = keep nothing */
+    int32_t fused_cluster;      /* METASD_PATH_FUSED: CTAs per cluster (0 = the smallest that fits) */
+    int32_t fused_threads;      /* METASD_PATH_FUSED: threads per CTA (0 = chosen from the slice length) */
+    int32_t wait_poll_limit;    /* polls after which a device-side wait on an asynchronous copy gives up and sets
+                                   METASD_STATUS_TIMEOUT (0 = about a quarter of a second).  For tests of that path. */
+    int32_t reserved;           /* must be 0 */
 } metasd_config;
 
 /* Optional per-position diagnostics of metasd_verify, [B, k]. */
@@ -125,8 +150,8 @@ int metasd_init(metasd_ctx **out, const metasd_config *cfg);
 /* Frees everything metasd_init allocated.  NULL is accepted. */
 void metasd_destroy(metasd_ctx *ctx);
 
-/* Per-query re-initialisation ("the bandit is re-initialised for every new query", experimental
- * setup): t <- 0 and cleared arm statistics for the n sequences listed in seq_ids (device int32),
+/* Per-query re-initialisation (experimental setup section: one bandit run per query):
+ * t <- 0 and cleared arm statistics for the n sequences listed in seq_ids (device int32),
  * or for all sequences when seq_ids is NULL.  Ids outside [0, max_batch) are ignored. */
 int metasd_reset(metasd_ctx *ctx, const int32_t *seq_ids, int32_t n, void *stream);
 
@@ -192,6 +217,13 @@ size_t metasd_state_bytes(const metasd_ctx *ctx);
 int metasd_state_export(metasd_ctx *ctx, void *host_buf, size_t bytes, void *stream);
 int metasd_state_import(metasd_ctx *ctx, const void *host_buf, size_t bytes, void *stream);
 
+/* The check metasd_state_import makes before anything reaches the device, as a host-only call (no CUDA): the header
+ * must match cfg, every round counter must be >= 0, every current arm and every arm recorded in an SW-UCB window
+ * must lie in [0, K), every statistic must be finite and every count non-negative -- the kernels index and divide
+ * with these values.  Returns METASD_OK, METASD_ERR_BAD_STATE_BLOB, or METASD_ERR_INVALID_ARGUMENT (NULL, short
+ * buffer, invalid cfg). */
+int metasd_state_validate(const metasd_config *cfg, const void *host_buf, size_t bytes);
+
 /* Reads and clears the status word (synchronises the stream).  Defined outputs: a non-finite row
  * pair is rejected with d_TV = 1; an out-of-range token is rejected; q(x) = 0 < p(x) is accepted. */
 int metasd_last_status(metasd_ctx *ctx, uint32_t *host_flags, void *stream);
@@ -203,6 +235,10 @@ uint64_t metasd_kernel_launches(const metasd_ctx *ctx);
  * (METASD_PATH_STREAMING or METASD_PATH_FUSED). */
 int metasd_resolved_path(const metasd_ctx *ctx, int32_t k);
 
+/* The row-statistics variant the streaming path of this context launches for 16-byte aligned rows
+ * (a metasd_row_kernel other than METASD_ROWS_AUTO). */
+int metasd_resolved_row_kernel(const metasd_ctx *ctx);
+
 /* One verification round for callers that cannot allocate device memory.  (The paper has no
  * counterpart: this is a packaging of the stateless part of metasd_verify -- Algorithm 4's verification loop
  * and the reward -- for hosts where cudaMalloc is not available to this code: a serving process whose
@@ -210,7 +246,8 @@ int metasd_resolved_path(const metasd_ctx *ctx, int32_t k);
  * latency-critical thread that must stay clear of the allocator.  Such callers cannot create a
  * context, so there is no bandit here and nothing persists between calls.)
  *
- * The scratch of the two kernels lives in a fixed array inside the library image (about 0.7 MB, held
+ * It launches the kernels of a default streaming context (the staged row-statistics kernel for 16-byte aligned
+ * rows, the plain-load one otherwise, then the epilogue).  Their scratch lives in a fixed array inside the library image (about 0.7 MB, held
  * by every GPU that loads the library until the process exits), which bounds the sizes:
  * batch <= METASD_NOALLOC_MAX_BATCH and batch * (k + 1) <= METASD_NOALLOC_MAX_ROWS; beyond that the
  * call returns METASD_ERR_UNSUPPORTED and launches nothing.  The call makes no cudaMalloc / cudaFree

@@ -20,6 +20,7 @@ BF16, FP32 = 0, 1
 UCB, DUCB, SWUCB, EXP3, RAND, PETC = 0, 1, 2, 3, 4, 5
 REWARD_BD, REWARD_BE = 0, 1
 PATH_AUTO, PATH_STREAMING, PATH_FUSED = 0, 1, 2
+ROWS_AUTO, ROWS_PLAIN, ROWS_STAGED, ROWS_BULK = 0, 1, 2, 3
 STATUS_NONFINITE, STATUS_TOKEN_OOR, STATUS_Q_ZERO, STATUS_TIMEOUT, STATUS_BAD_POINTER, STATUS_BAD_LENGTH = 1, 2, 4, 8, 16, 32
 
 OK, ERR_INVALID_ARGUMENT, ERR_UNSUPPORTED, ERR_CUDA, ERR_NO_MEMORY, ERR_BAD_STATE_BLOB = 0, -1, -2, -3, -4, -5
@@ -31,7 +32,8 @@ EXPORTS = (
     "metasd_default_config", "metasd_init", "metasd_destroy", "metasd_reset", "metasd_select",
     "metasd_verify", "metasd_verify_host", "metasd_state_bytes", "metasd_state_export",
     "metasd_state_import", "metasd_last_status", "metasd_kernel_launches", "metasd_resolved_path",
-    "metasd_strerror", "metasd_verify_noalloc", "metasd_set_draft_lengths",
+    "metasd_strerror", "metasd_verify_noalloc", "metasd_set_draft_lengths", "metasd_state_validate",
+    "metasd_resolved_row_kernel",
 )
 
 
@@ -43,6 +45,9 @@ class MetasdConfig(C.Structure):
         ("reward", C.c_int32), ("window", C.c_int32), ("device", C.c_int32), ("path", C.c_int32),
         ("sequence_base", C.c_uint32), ("host_staging", C.c_int32),
         ("beta", C.c_double), ("gamma", C.c_double), ("reward_temperature", C.c_double),
+        ("row_kernel", C.c_int32), ("row_threads", C.c_int32), ("row_stages", C.c_int32),
+        ("keep_permille", C.c_int32), ("fused_cluster", C.c_int32), ("fused_threads", C.c_int32),
+        ("wait_poll_limit", C.c_int32), ("reserved", C.c_int32),
     ]
 
 
@@ -91,6 +96,8 @@ def load_library(path: Optional[str] = None):
     lib.metasd_set_draft_lengths.argtypes = [vp, vp]
     lib.metasd_kernel_launches.restype = u64
     lib.metasd_resolved_path.argtypes = [vp, i32]
+    lib.metasd_resolved_row_kernel.argtypes = [vp]
+    lib.metasd_state_validate.argtypes = [C.POINTER(MetasdConfig), vp, C.c_size_t]
     lib.metasd_verify_noalloc.argtypes = [i32, i32, i32, i32, vp, vp, vp, C.c_float, C.c_float, i32, u64, C.c_uint32,
                                           C.c_uint32, vp, vp, vp, vp, vp]
     lib.metasd_strerror.argtypes = [C.c_int]
@@ -142,7 +149,9 @@ class MetaSD:
     def __init__(self, max_batch: int, n_drafters: int, max_draft: int, vocab: int, dtype="bf16",
                  bandit="ucb", beta: float = 0.01, gamma: float = 0.975, window: int = 50,
                  reward: int = REWARD_BD, reward_temperature: float = 1.0, device: int = 0,
-                 path: int = PATH_AUTO, sequence_base: int = 0, host_staging: bool = False):
+                 path: int = PATH_AUTO, sequence_base: int = 0, host_staging: bool = False, **tuning):
+        """tuning: the configuration's tuning and test fields by name (row_kernel, row_threads, row_stages,
+        keep_permille, fused_cluster, fused_threads, wait_poll_limit)."""
         self.lib = load_library()
         cfg = default_config()
         cfg.max_batch, cfg.n_drafters, cfg.max_draft, cfg.vocab = max_batch, n_drafters, max_draft, vocab
@@ -152,6 +161,11 @@ class MetaSD:
         cfg.reward, cfg.reward_temperature = reward, reward_temperature
         cfg.device, cfg.path, cfg.sequence_base = device, path, sequence_base
         cfg.host_staging = 1 if host_staging else 0
+        for name, value in tuning.items():
+            if name not in ("row_kernel", "row_threads", "row_stages", "keep_permille", "fused_cluster",
+                            "fused_threads", "wait_poll_limit"):
+                raise TypeError("unknown configuration field %r" % name)
+            setattr(cfg, name, int(value))
         self.cfg = cfg
         self.device = torch.device("cuda", device)
         self._ctx = C.c_void_p()
@@ -246,6 +260,9 @@ class MetaSD:
     def resolved_path(self, k: int) -> int:
         return int(self.lib.metasd_resolved_path(self._ctx, k))
 
+    def resolved_row_kernel(self) -> int:
+        return int(self.lib.metasd_resolved_row_kernel(self._ctx))
+
 
 def verify_noalloc(target_logits: torch.Tensor, draft_logits: torch.Tensor, draft_tokens: torch.Tensor,
                    temperature: float, seed: int, round_: int, accepted_len: torch.Tensor,
@@ -260,6 +277,12 @@ def verify_noalloc(target_logits: torch.Tensor, draft_logits: torch.Tensor, draf
         C.c_float(temperature), C.c_float(reward_temperature), reward_kind, C.c_uint64(seed),
         C.c_uint32(sequence_base), C.c_uint32(round_), _ptr(accepted_len), _ptr(next_token), _ptr(reward),
         _ptr(status), _stream(dev))
+
+
+def state_validate(cfg: MetasdConfig, blob: bytes) -> int:
+    """metasd_state_validate: the host-only check of a state blob (returns the library's error code)."""
+    buf = C.create_string_buffer(blob, len(blob))
+    return int(load_library().metasd_state_validate(C.byref(cfg), buf, len(blob)))
 
 
 def pointer_table(tensors: Sequence[torch.Tensor]) -> torch.Tensor:

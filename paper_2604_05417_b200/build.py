@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmetasd.so")
-SOURCES = ["metasd_api.cu", "metasd_streaming.cu", "metasd_fused.cu", "metasd_noalloc.cu"]
+SOURCES = ["metasd_api.cu", "metasd_streaming.cu", "metasd_bulk.cu", "metasd_fused.cu", "metasd_noalloc.cu"]
 HEADERS = ["metasd_internal.h", "metasd_device.cuh", os.path.join(ROOT, "include", "metasd.h")]
 
 

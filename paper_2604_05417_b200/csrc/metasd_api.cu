@@ -15,7 +15,6 @@ struct metasd_ctx {
     BanditState st;
     RowStats *stats;     // scratch of the streaming path: [max_batch, max_draft + 1]
     uint32_t *status;    // device status word
-    const void **table_clean;   // the checked copy of the caller's drafter table (16 entries)
     const int32_t *draft_len;   // the caller's per-sequence draft lengths (device), or nullptr
     uint64_t launches;
     // staging for metasd_verify_host
@@ -24,13 +23,8 @@ struct metasd_ctx {
     float *stage_reward;
     bool fused_ready;
     FusedPlan plan;
-    int keep_permille;   // share of every row that the streaming kernel asks L2 to keep between its sweeps
-    int k1_stages;       // depth of the row-statistics kernel's cp.async pipeline (0 or 1: plain loads)
-    // split streaming path
-    int grp_size, grp_ctas;
-    GroupRecord *grp_rec;
-    double *grp_min;
-    uint32_t *grp_count;
+    RowGeometry geo;     // shape of the row-statistics launch
+    int keep_permille;   // share of every row that the row-statistics kernel asks L2 to keep between its sweeps
 };
 
 namespace {
@@ -42,6 +36,32 @@ struct BlobHeader {
 constexpr uint32_t BLOB_MAGIC = 0x4D534453u;  // "MSDS"
 
 size_t logit_size(int dtype) { return dtype == METASD_BF16 ? 2 : 4; }
+
+size_t blob_bytes(const metasd_config &c)
+{
+    const size_t B = c.max_batch, K = c.n_drafters, tau = c.window;
+    return sizeof(BlobHeader) + 2 * B * sizeof(int32_t) + 2 * B * K * sizeof(double) + B * tau * sizeof(int32_t) +
+           B * tau * sizeof(double);
+}
+
+// Makes the context's device current for the lifetime of the object and restores the caller's on the way out.
+struct DeviceScope {
+    int previous = -1;
+    cudaError_t error = cudaSuccess;
+    explicit DeviceScope(int device)
+    {
+        error = cudaGetDevice(&previous);
+        if (error == cudaSuccess && previous != device) error = cudaSetDevice(device);
+        else if (error == cudaSuccess) previous = -1;   // nothing to restore
+    }
+    ~DeviceScope()
+    {
+        if (previous >= 0) cudaSetDevice(previous);
+    }
+};
+#define ON_DEVICE_OF(ctx)                                   \
+    DeviceScope scope_((ctx)->cfg.device);                  \
+    if (scope_.error != cudaSuccess) return cuda_fail(scope_.error)
 
 int cuda_fail(cudaError_t e) { return e == cudaErrorMemoryAllocation ? METASD_ERR_NO_MEMORY : METASD_ERR_CUDA; }
 
@@ -67,6 +87,11 @@ int validate_config(const metasd_config *c)
     if (!(c->beta >= 0.0) || !isfinite(c->beta)) return METASD_ERR_INVALID_ARGUMENT;
     if (!(c->gamma > 0.0) || !(c->gamma <= 1.0)) return METASD_ERR_INVALID_ARGUMENT;
     if (!(c->reward_temperature > 0.0) || !isfinite(c->reward_temperature)) return METASD_ERR_INVALID_ARGUMENT;
+    if (c->row_kernel < METASD_ROWS_AUTO || c->row_kernel > METASD_ROWS_BULK) return METASD_ERR_UNSUPPORTED;
+    if (c->row_threads < 0 || c->row_stages < 0 || c->keep_permille > 1000) return METASD_ERR_INVALID_ARGUMENT;
+    if (c->fused_cluster < 0 || c->fused_cluster > 16 || c->fused_threads < 0 || c->fused_threads % 32 != 0)
+        return METASD_ERR_INVALID_ARGUMENT;
+    if (c->wait_poll_limit < 0 || c->reserved != 0) return METASD_ERR_INVALID_ARGUMENT;
     if ((uint64_t)c->vocab * (uint64_t)(c->max_draft + 1) >= (1ull << 31)) return METASD_ERR_UNSUPPORTED;
     return METASD_OK;
 }
@@ -77,10 +102,45 @@ void free_all(metasd_ctx *c)
     cudaFree(c->st.win_arm); cudaFree(c->st.win_reward); cudaFree(c->stats); cudaFree(c->status);
     cudaFree(c->stage_target); cudaFree(c->stage_draft); cudaFree(c->stage_tokens);
     cudaFree(c->stage_acc); cudaFree(c->stage_tok); cudaFree(c->stage_reward);
-    cudaFree(c->grp_rec); cudaFree(c->grp_min); cudaFree(c->grp_count);
 }
 
 }  // namespace
+
+// Everything of a blob's payload that a kernel later uses as an index or divides by: round counters, arms, the arms
+// in the SW-UCB windows, and finite, non-negative statistics.  Plain host code: no CUDA call.
+int metasd::validate_state_payload(const metasd_config &cfg, const void *payload)
+{
+    const size_t B = cfg.max_batch, K = cfg.n_drafters, tau = cfg.window;
+    const char *r = (const char *)payload;
+    auto take = [&](void *dst, size_t n) { memcpy(dst, r, n); r += n; };
+    for (size_t i = 0; i < B; ++i) {
+        int32_t t;
+        take(&t, sizeof t);
+        if (t < 0 || t >= 0x7FFFFFF0) return METASD_ERR_BAD_STATE_BLOB;
+    }
+    for (size_t i = 0; i < B; ++i) {
+        int32_t arm;
+        take(&arm, sizeof arm);
+        if (arm < 0 || arm >= (int32_t)K) return METASD_ERR_BAD_STATE_BLOB;
+    }
+    for (size_t i = 0; i < 2 * B * K; ++i) {   // stat_a (means, sums, weights), stat_b (counts, memberships)
+        double x;
+        take(&x, sizeof x);
+        if (!isfinite(x) || (i >= B * K && x < 0.0)) return METASD_ERR_BAD_STATE_BLOB;
+        if (cfg.bandit == METASD_EXP3 && i < B * K && x < 0.0) return METASD_ERR_BAD_STATE_BLOB;
+    }
+    for (size_t i = 0; i < B * tau; ++i) {
+        int32_t arm;
+        take(&arm, sizeof arm);
+        if (arm < 0 || arm >= (int32_t)K) return METASD_ERR_BAD_STATE_BLOB;
+    }
+    for (size_t i = 0; i < B * tau; ++i) {
+        double x;
+        take(&x, sizeof x);
+        if (!isfinite(x)) return METASD_ERR_BAD_STATE_BLOB;
+    }
+    return METASD_OK;
+}
 
 extern "C" {
 
@@ -113,7 +173,6 @@ int metasd_init(metasd_ctx **out, const metasd_config *cfg)
     if (rc != METASD_OK) return rc;
     int n_dev = 0;
     if (cudaGetDeviceCount(&n_dev) != cudaSuccess || cfg->device >= n_dev) return METASD_ERR_CUDA;
-    CK(cudaSetDevice(cfg->device));
     if (cfg->path == METASD_PATH_FUSED && !fused_supported(cfg->logit_dtype, cfg->vocab, cfg->max_draft))
         return METASD_ERR_UNSUPPORTED;
 
@@ -121,16 +180,11 @@ int metasd_init(metasd_ctx **out, const metasd_config *cfg)
     if (!c) return METASD_ERR_NO_MEMORY;
     memset(c, 0, sizeof *c);
     c->cfg = *cfg;
-    {   // the best measured values on B200 for 128k-152k vocabularies (METASD_KEEP_PERMILLE overrides, for tuning)
-        const char *kp = getenv("METASD_KEEP_PERMILLE");
-        const int v = kp && *kp ? atoi(kp) : (cfg->logit_dtype == METASD_BF16 ? 750 : 900);
-        c->keep_permille = v < 0 ? 0 : (v > 1000 ? 1000 : v);
-    }
-    {
-        // 4: rows staged through shared memory; 0 (METASD_K1_STAGES=0, for comparison): plain loads
-        const char *ks = getenv("METASD_K1_STAGES");
-        c->k1_stages = ks && *ks ? atoi(ks) : 4;
-    }
+    DeviceScope scope(cfg->device);
+    if (scope.error != cudaSuccess) { delete c; return cuda_fail(scope.error); }
+    // the share of a row that L2 is asked to keep: the best measured values on B200 for 128k-152k vocabularies
+    c->keep_permille = cfg->keep_permille == 0 ? (cfg->logit_dtype == METASD_BF16 ? 750 : 900)
+                                               : (cfg->keep_permille < 0 ? 0 : cfg->keep_permille);
     const size_t B = cfg->max_batch, K = cfg->n_drafters, tau = cfg->window, kp1 = cfg->max_draft + 1;
     cudaError_t e = cudaSuccess;
     auto alloc = [&](void **p, size_t bytes) {
@@ -144,7 +198,6 @@ int metasd_init(metasd_ctx **out, const metasd_config *cfg)
     alloc((void **)&c->st.win_reward, B * tau * sizeof(double));
     alloc((void **)&c->stats, B * kp1 * sizeof(RowStats));
     alloc((void **)&c->status, sizeof(uint32_t));
-    alloc((void **)&c->table_clean, 16 * sizeof(void *));
     if (cfg->host_staging) {
         const size_t row = (size_t)cfg->vocab * logit_size(cfg->logit_dtype);
         alloc(&c->stage_target, B * kp1 * row);
@@ -154,28 +207,24 @@ int metasd_init(metasd_ctx **out, const metasd_config *cfg)
         alloc((void **)&c->stage_tok, B * sizeof(int32_t));
         alloc((void **)&c->stage_reward, B * sizeof(float));
     }
+    bool unsupported = false;
     if (e == cudaSuccess) {
-        e = split_prepare(cfg->device, cfg->logit_dtype, cfg->vocab, &c->grp_ctas, &c->grp_size);
-        if (e == cudaSuccess && c->grp_size > 1) {
-            alloc((void **)&c->grp_rec, B * kp1 * c->grp_size * sizeof(GroupRecord));
-            alloc((void **)&c->grp_min, B * kp1 * c->grp_size * sizeof(double));
-            alloc((void **)&c->grp_count, B * kp1 * sizeof(uint32_t));
-        }
+        e = streaming_prepare(cfg->device, cfg->logit_dtype, *cfg, &c->geo);
+        if (e == cudaErrorNotSupported) { unsupported = true; (void)cudaGetLastError(); }
     }
     if (e == cudaSuccess) e = cudaMemset(c->status, 0, sizeof(uint32_t));
     if (e == cudaSuccess) e = launch_reset(c->st, cfg->max_batch, cfg->n_drafters, cfg->window, cfg->bandit, cfg->gamma,
                                             cfg->sequence_base, nullptr, cfg->max_batch, 0);
-    if (e == cudaSuccess && cfg->path == METASD_PATH_FUSED &&
-        fused_supported(cfg->logit_dtype, cfg->vocab, cfg->max_draft)) {
-        e = fused_prepare(cfg->device, cfg->logit_dtype, cfg->vocab, cfg->max_batch, &c->plan);
+    if (e == cudaSuccess && cfg->path == METASD_PATH_FUSED) {
+        e = fused_prepare(cfg->device, cfg->logit_dtype, cfg->vocab, cfg->max_batch, cfg->fused_cluster, cfg->fused_threads,
+                          &c->plan);
         c->fused_ready = (e == cudaSuccess);
-        if (cfg->path == METASD_PATH_AUTO && e != cudaSuccess) { (void)cudaGetLastError(); e = cudaSuccess; }
     }
     if (e == cudaSuccess) e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {
         free_all(c);
         delete c;
-        return cuda_fail(e);
+        return unsupported ? METASD_ERR_UNSUPPORTED : cuda_fail(e);
     }
     *out = c;
     return METASD_OK;
@@ -184,14 +233,17 @@ int metasd_init(metasd_ctx **out, const metasd_config *cfg)
 void metasd_destroy(metasd_ctx *ctx)
 {
     if (!ctx) return;
-    cudaSetDevice(ctx->cfg.device);
-    free_all(ctx);
+    {
+        DeviceScope scope(ctx->cfg.device);
+        free_all(ctx);
+    }
     delete ctx;
 }
 
 int metasd_reset(metasd_ctx *ctx, const int32_t *seq_ids, int32_t n, void *stream)
 {
     if (!ctx || n < 0) return METASD_ERR_INVALID_ARGUMENT;
+    ON_DEVICE_OF(ctx);
     if (!seq_ids) n = ctx->cfg.max_batch;
     CK(launch_reset(ctx->st, ctx->cfg.max_batch, ctx->cfg.n_drafters, ctx->cfg.window, ctx->cfg.bandit, ctx->cfg.gamma,
                     ctx->cfg.sequence_base, seq_ids, n, (cudaStream_t)stream));
@@ -202,8 +254,9 @@ int metasd_reset(metasd_ctx *ctx, const int32_t *seq_ids, int32_t n, void *strea
 int metasd_select(metasd_ctx *ctx, int32_t batch, int32_t *arm_out, void *stream)
 {
     if (!ctx || !arm_out || batch < 1 || batch > ctx->cfg.max_batch) return METASD_ERR_INVALID_ARGUMENT;
-    CK(launch_select(ctx->st, batch, arm_out, (cudaStream_t)stream));
-    ctx->launches += 1;
+    ON_DEVICE_OF(ctx);
+    // the arm of the coming round was chosen at the end of the previous epilogue: the call is a copy
+    CK(cudaMemcpyAsync(arm_out, ctx->st.arm, (size_t)batch * sizeof(int32_t), cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
     return METASD_OK;
 }
 
@@ -217,6 +270,8 @@ int metasd_resolved_path(const metasd_ctx *ctx, int32_t k)
     return METASD_PATH_STREAMING;
 }
 
+int metasd_resolved_row_kernel(const metasd_ctx *ctx) { return ctx ? ctx->geo.kernel : METASD_ERR_INVALID_ARGUMENT; }
+
 int metasd_verify(metasd_ctx *ctx, int32_t batch, int32_t k, const void *target_logits, const void *draft_logits,
                   const void *const *drafter_ptrs, const int32_t *draft_tokens, int64_t token_arm_stride,
                   float temperature, uint64_t seed, int32_t *accepted_len, int32_t *next_token, float *reward,
@@ -228,6 +283,9 @@ int metasd_verify(metasd_ctx *ctx, int32_t batch, int32_t k, const void *target_
     if (!target_logits || !draft_tokens || !accepted_len || !next_token || !reward) return METASD_ERR_INVALID_ARGUMENT;
     if ((draft_logits == nullptr) == (drafter_ptrs == nullptr)) return METASD_ERR_INVALID_ARGUMENT;
     if (!(temperature >= 0.f) || !isfinite(temperature) || token_arm_stride < 0) return METASD_ERR_INVALID_ARGUMENT;
+    const int path = metasd_resolved_path(ctx, k);
+    if (ctx->draft_len && cfg.path == METASD_PATH_FUSED) return METASD_ERR_UNSUPPORTED;
+    ON_DEVICE_OF(ctx);
 
     VerifyParams p;
     memset(&p, 0, sizeof p);
@@ -243,36 +301,25 @@ int metasd_verify(metasd_ctx *ctx, int32_t batch, int32_t k, const void *target_
     p.seed = seed; p.beta = cfg.beta; p.gamma = cfg.gamma;
     p.accepted_len = accepted_len; p.next_token = next_token; p.reward = reward; p.diag = diag;
     p.st = ctx->st; p.stats = ctx->stats; p.status = ctx->status;
-    p.keep_permille = ctx->keep_permille;
     {
         const long long nvec = (long long)cfg.vocab * (long long)logit_size(cfg.logit_dtype) / 16;
         p.keep_from_vec = (int32_t)(nvec - nvec * ctx->keep_permille / 1000);
     }
-    p.k1_stages = ctx->k1_stages;
-    p.grp_size = ctx->grp_size; p.grp_ctas = ctx->grp_ctas;
-    p.grp_rec = ctx->grp_rec; p.grp_min = ctx->grp_min; p.grp_count = ctx->grp_count;
+    p.poll_limit = cfg.wait_poll_limit > 0 ? (uint32_t)cfg.wait_poll_limit : (1u << 22);
     const size_t row_bytes = (size_t)cfg.vocab * logit_size(cfg.logit_dtype);
-    // with a pointer table the per-drafter bases are not visible here: the caller's contract is that
-    // they are aligned like the target
+    // with a pointer table the per-drafter bases are not visible here: the kernels check every entry they use
+    // against table_mask and never dereference one that fails
     p.vector_ok = row_bytes % 16 == 0 && ((uintptr_t)target_logits % 16) == 0 &&
                   (draft_logits ? ((uintptr_t)draft_logits % 16) == 0 : 1);
+    p.table_mask = p.vector_ok ? 15u : (uint32_t)(logit_size(cfg.logit_dtype) - 1);
 
     cudaError_t e;
-    if (drafter_ptrs && metasd_resolved_path(ctx, k) != METASD_PATH_FUSED) {   // the fused kernel checks for itself
-        const uint32_t mask = p.vector_ok ? 15u : (uint32_t)(logit_size(cfg.logit_dtype) - 1);
-        e = launch_sanitize_table(drafter_ptrs, cfg.n_drafters, target_logits, mask, ctx->table_clean, ctx->status,
-                                  (cudaStream_t)stream);
-        if (e != cudaSuccess) return cuda_fail(e);
-        ctx->launches += 1;
-        p.drafter_ptrs = ctx->table_clean;
-    }
-    if (ctx->draft_len && cfg.path == METASD_PATH_FUSED) return METASD_ERR_UNSUPPORTED;
-    if (metasd_resolved_path(ctx, k) == METASD_PATH_FUSED && p.vector_ok)
+    if (path == METASD_PATH_FUSED && p.vector_ok)
         e = launch_fused(p, cfg.logit_dtype, ctx->plan, (cudaStream_t)stream, &ctx->launches);
     else if (cfg.path == METASD_PATH_FUSED)
         return METASD_ERR_UNSUPPORTED;
     else
-        e = launch_streaming(p, cfg.logit_dtype, (cudaStream_t)stream, &ctx->launches);
+        e = launch_streaming(p, cfg.logit_dtype, ctx->geo, (cudaStream_t)stream, &ctx->launches);
     return e == cudaSuccess ? METASD_OK : cuda_fail(e);
 }
 
@@ -289,6 +336,7 @@ int metasd_verify_host(metasd_ctx *ctx, int32_t batch, int32_t k, const void *ho
                        int32_t *host_arm_next, void *stream)
 {
     if (!ctx || !ctx->stage_target) return METASD_ERR_INVALID_ARGUMENT;
+    ON_DEVICE_OF(ctx);
     const metasd_config &cfg = ctx->cfg;
     if (batch < 1 || batch > cfg.max_batch || k < 1 || k > cfg.max_draft) return METASD_ERR_INVALID_ARGUMENT;
     if (!host_target_logits || !host_draft_logits || !host_draft_tokens || !host_accepted_len || !host_next_token ||
@@ -311,17 +359,12 @@ int metasd_verify_host(metasd_ctx *ctx, int32_t batch, int32_t k, const void *ho
     return METASD_OK;
 }
 
-size_t metasd_state_bytes(const metasd_ctx *ctx)
-{
-    if (!ctx) return 0;
-    const size_t B = ctx->cfg.max_batch, K = ctx->cfg.n_drafters, tau = ctx->cfg.window;
-    return sizeof(BlobHeader) + 2 * B * sizeof(int32_t) + 2 * B * K * sizeof(double) + B * tau * sizeof(int32_t) +
-           B * tau * sizeof(double);
-}
+size_t metasd_state_bytes(const metasd_ctx *ctx) { return ctx ? blob_bytes(ctx->cfg) : 0; }
 
 int metasd_state_export(metasd_ctx *ctx, void *host_buf, size_t bytes, void *stream)
 {
     if (!ctx || !host_buf || bytes < metasd_state_bytes(ctx)) return METASD_ERR_INVALID_ARGUMENT;
+    ON_DEVICE_OF(ctx);
     const size_t B = ctx->cfg.max_batch, K = ctx->cfg.n_drafters, tau = ctx->cfg.window;
     cudaStream_t s = (cudaStream_t)stream;
     BlobHeader h = {BLOB_MAGIC, 1u, ctx->cfg.max_batch, ctx->cfg.n_drafters, ctx->cfg.window, ctx->cfg.bandit};
@@ -343,17 +386,30 @@ int metasd_state_export(metasd_ctx *ctx, void *host_buf, size_t bytes, void *str
     return METASD_OK;
 }
 
+int metasd_state_validate(const metasd_config *cfg, const void *host_buf, size_t bytes)
+{
+    int rc = validate_config(cfg);
+    if (rc != METASD_OK) return rc;
+    if (!host_buf || bytes < blob_bytes(*cfg)) return METASD_ERR_INVALID_ARGUMENT;
+    BlobHeader h;
+    memcpy(&h, host_buf, sizeof h);
+    if (h.magic != BLOB_MAGIC || h.version != 1u || h.max_batch != cfg->max_batch || h.n_drafters != cfg->n_drafters ||
+        h.window != cfg->window || h.bandit != cfg->bandit)
+        return METASD_ERR_BAD_STATE_BLOB;
+    return validate_state_payload(*cfg, (const char *)host_buf + sizeof h);
+}
+
 int metasd_state_import(metasd_ctx *ctx, const void *host_buf, size_t bytes, void *stream)
 {
     if (!ctx || !host_buf || bytes < metasd_state_bytes(ctx)) return METASD_ERR_INVALID_ARGUMENT;
-    BlobHeader h;
-    memcpy(&h, host_buf, sizeof h);
-    if (h.magic != BLOB_MAGIC || h.version != 1u || h.max_batch != ctx->cfg.max_batch ||
-        h.n_drafters != ctx->cfg.n_drafters || h.window != ctx->cfg.window || h.bandit != ctx->cfg.bandit)
-        return METASD_ERR_BAD_STATE_BLOB;
+    // the kernels index with what the blob holds (arms, window entries, round counters): nothing reaches the device
+    // before every value has been checked on the host
+    int rc = metasd_state_validate(&ctx->cfg, host_buf, bytes);
+    if (rc != METASD_OK) return rc;
+    ON_DEVICE_OF(ctx);
     const size_t B = ctx->cfg.max_batch, K = ctx->cfg.n_drafters, tau = ctx->cfg.window;
     cudaStream_t s = (cudaStream_t)stream;
-    const char *r = (const char *)host_buf + sizeof h;
+    const char *r = (const char *)host_buf + sizeof(BlobHeader);
     auto push = [&](void *dst, size_t n) -> cudaError_t {
         cudaError_t e = cudaMemcpyAsync(dst, r, n, cudaMemcpyHostToDevice, s);
         r += n;
@@ -372,6 +428,7 @@ int metasd_state_import(metasd_ctx *ctx, const void *host_buf, size_t bytes, voi
 int metasd_last_status(metasd_ctx *ctx, uint32_t *host_flags, void *stream)
 {
     if (!ctx || !host_flags) return METASD_ERR_INVALID_ARGUMENT;
+    ON_DEVICE_OF(ctx);
     cudaStream_t s = (cudaStream_t)stream;
     CK(cudaMemcpyAsync(host_flags, ctx->status, sizeof(uint32_t), cudaMemcpyDeviceToHost, s));
     CK(cudaMemsetAsync(ctx->status, 0, sizeof(uint32_t), s));
@@ -389,7 +446,7 @@ const char *metasd_strerror(int code)
     case METASD_ERR_UNSUPPORTED: return "unsupported configuration";
     case METASD_ERR_CUDA: return "CUDA error (no device, or a runtime call failed)";
     case METASD_ERR_NO_MEMORY: return "out of memory";
-    case METASD_ERR_BAD_STATE_BLOB: return "state blob does not match this context";
+    case METASD_ERR_BAD_STATE_BLOB: return "state blob does not match this context or holds values outside their range";
     default: return "unknown error";
     }
 }

@@ -93,6 +93,19 @@ __device__ __forceinline__ int drafted(const int32_t *draft_len, int b, int k)
     return kb < 1 ? 1 : (kb > k ? k : kb);
 }
 
+// Rows of the drafter sequence b plays: the gathered tensor, or the entry of the caller's pointer table for the
+// sequence's arm.  An entry that is NULL or not aligned like the target (table_mask: 15 on the vector path, else
+// the element size minus one) is never dereferenced: the target tensor stands in for it, so that the outputs of the
+// sequences that play that drafter are defined (if meaningless); the epilogue flags such a table once per call.
+template <typename LT>
+__device__ __forceinline__ const LT *draft_rows(const VerifyParams &p, int b)
+{
+    if (p.draft) return reinterpret_cast<const LT *>(p.draft);
+    const void *q = p.drafter_ptrs[p.st.arm[b]];
+    if (q == nullptr || (reinterpret_cast<uintptr_t>(q) & p.table_mask) != 0) q = p.target;
+    return reinterpret_cast<const LT *>(q);
+}
+
 // Streaming 16-byte load that does not allocate in L1.
 __device__ __forceinline__ uint4 ld_stream(const void *p)
 {
@@ -278,6 +291,18 @@ __device__ __forceinline__ void bulk_load(void *dst, const void *src, uint32_t b
                  ::"r"(smem_addr(dst)), "l"(src), "r"(bytes), "r"(smem_addr(bar))
                  : "memory");
 }
+
+// 16 bytes from this CTA's shared memory.
+__device__ __forceinline__ uint4 lds16(uint32_t addr)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+    return v;
+}
+
+// Programmatic dependent launch: lets the next kernel in the stream be set up while this grid still runs.  That
+// kernel waits for this whole grid (griddepcontrol.wait) before it touches anything this one reads or writes.
+__device__ __forceinline__ void launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 __device__ __forceinline__ float warp_sum_f(float v)
 {

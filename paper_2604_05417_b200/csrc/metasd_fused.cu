@@ -18,8 +18,6 @@
 // Rank 0 of the cluster then writes the outputs, forms the reward, and one warp updates the bandit and
 // selects the next arm with one lane per drafter (Algorithm 2, update and selection steps).
 #include <limits.h>
-#include <stdio.h>
-#include <stdlib.h>
 
 #include "metasd_device.cuh"
 
@@ -821,12 +819,6 @@ bool geometry(int dtype, int V, int C, int smem_per_sm, FusedPlan *pl)
     return true;
 }
 
-int env_int(const char *name, int fallback)
-{
-    const char *s = getenv(name);
-    return s && *s ? atoi(s) : fallback;
-}
-
 }  // namespace
 
 bool fused_supported(int dtype, int V, int k)
@@ -840,8 +832,8 @@ bool fused_supported(int dtype, int V, int k)
 
 // Chooses the cluster size for this device: the smallest for which two CTAs fit an SM, and asks the occupancy
 // calculator how many clusters are co-resident (GPC shapes decide).
-// METASD_FUSED_CLUSTER / METASD_FUSED_THREADS (environment) pin the choice for tuning runs.
-cudaError_t fused_prepare(int device, int dtype, int V, int max_batch, FusedPlan *plan)
+// pin_c / pin_t (the configuration's fused_cluster / fused_threads; 0 = free) pin the choice for tuning runs.
+cudaError_t fused_prepare(int device, int dtype, int V, int max_batch, int pin_c, int pin_t, FusedPlan *plan)
 {
     plan->cluster = 0;
     int smem_per_sm = 0;
@@ -852,7 +844,6 @@ cudaError_t fused_prepare(int device, int dtype, int V, int max_batch, FusedPlan
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
     if (e != cudaSuccess) return e;
-    const int pin_c = env_int("METASD_FUSED_CLUSTER", 0), pin_t = env_int("METASD_FUSED_THREADS", 0);
     double best = 0.0;
     for (int C = 1; C <= FUSED_MAX_CLUSTER; ++C) {
         if (pin_c && C != pin_c) continue;
@@ -881,9 +872,6 @@ cudaError_t fused_prepare(int device, int dtype, int V, int max_batch, FusedPlan
         if (!plan->cluster || cost < best) { *plan = pl; best = cost; }
         if (!pin_c) break;   // the smallest size that fits: the largest slices, the fewest exchange partners
     }
-    if (plan->cluster && env_int("METASD_FUSED_VERBOSE", 0))
-        fprintf(stderr, "metasd fused plan: V=%d cluster=%d threads=%d vectors/cta=%d (chunks of %d), %zu B shared, %d clusters co-resident\n",
-                V, plan->cluster, plan->threads, plan->n_vec_cta, 1 << plan->n_slot, plan->smem_bytes, plan->max_clusters);
     return plan->cluster ? cudaSuccess : cudaErrorNotSupported;
 }
 

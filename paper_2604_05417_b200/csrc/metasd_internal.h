@@ -13,17 +13,10 @@ namespace metasd {
 struct RowStats {
     float max_a, sum_a;   // target row
     float max_b, sum_b;   // draft row (unused at the bonus position); max_b is the reference sum_b is relative to:
-                          // the row's maximum, or the target row's where the staged kernel could share it
+                          // the row's maximum, or the target row's where the staged kernels could share it
     double sum_min;       // sum_v min(p_v, q_v) = 1 - d_TV(p, q)
     int32_t argmax_a;     // first index of the target row's maximum
     uint32_t flags;       // METASD_STATUS_* of this row pair
-};
-
-// What one CTA of a group publishes about its part of a row pair (split streaming path).
-struct GroupRecord {
-    float max_a, sum_a, max_b, sum_b;
-    int32_t argmax_a;
-    int32_t pad[3];
 };
 
 // Bandit state of all sequences, structure of arrays in device memory.
@@ -34,6 +27,15 @@ struct BanditState {
     double *stat_b;      // [B, K] UCB: n;       D-UCB: discounted count
     int32_t *win_arm;    // [B, tau] SW-UCB: arm of round s in slot s mod tau
     double *win_reward;  // [B, tau]
+};
+
+// Shape of the row-statistics launch, resolved from the configuration once per context.
+struct RowGeometry {
+    int32_t kernel;     // metasd_row_kernel, never AUTO
+    int32_t threads;    // threads per CTA
+    int32_t stages;     // staging depth (0 for plain loads)
+    int32_t per_sm;     // CTAs per SM the shape is built for
+    int32_t n_sm;       // SMs of the device (persistent kernels size their grid with it)
 };
 
 struct VerifyParams {
@@ -63,19 +65,17 @@ struct VerifyParams {
     RowStats *stats;   // [batch, k+1]
     uint32_t *status;
     int32_t vector_ok; // rows are 16-byte aligned and a whole number of 16-byte vectors
-    int32_t keep_permille;   // share of every row (its end) that the first sweep asks L2 to keep
-    int32_t keep_from_vec;   // the same as an index: first 16-byte vector of a row in the kept share
-    int32_t k1_stages;       // depth of the row-statistics kernel's cp.async pipeline (0 or 1: plain loads)
-    // split streaming path: grp_size CTAs share a row pair (0: one CTA per row pair)
-    int32_t grp_size;
-    int32_t grp_ctas;        // CTAs of the launch (co-resident)
-    GroupRecord *grp_rec;    // [batch * (k + 1), grp_size]
-    double *grp_min;         // [batch * (k + 1), grp_size] partial sums of min(p, q)
-    uint32_t *grp_count;     // [batch * (k + 1)] arrivals, cleared before every launch
+    int32_t keep_from_vec;   // first 16-byte vector of a row in the share that the first sweep asks L2 to keep
+    uint32_t poll_limit;     // polls after which a wait on an asynchronous copy gives up
+    uint32_t table_mask;     // pointer-table mode: low address bits that must be clear in every entry
 };
 
-// streaming path (metasd_streaming.cu)
-cudaError_t launch_streaming(const VerifyParams &p, int dtype, cudaStream_t stream, uint64_t *launches);
+// streaming path (metasd_streaming.cu, metasd_bulk.cu)
+cudaError_t streaming_prepare(int device, int dtype, const metasd_config &cfg, RowGeometry *geo);
+cudaError_t launch_streaming(const VerifyParams &p, int dtype, const RowGeometry &geo, cudaStream_t stream, uint64_t *launches);
+bool bulk_shape_built(int threads, int stages);
+cudaError_t bulk_prepare(int dtype, RowGeometry *geo);
+cudaError_t launch_row_stats_bulk(const VerifyParams &p, int dtype, const RowGeometry &geo, cudaStream_t stream);
 // fused cluster path (metasd_fused.cu)
 struct FusedPlan {
     int32_t cluster;       // CTAs per cluster (0: no plan)
@@ -89,18 +89,14 @@ struct FusedPlan {
     long work_per_item;    // threads x vectors per thread
 };
 bool fused_supported(int dtype, int V, int k);
-cudaError_t fused_prepare(int device, int dtype, int V, int max_batch, FusedPlan *plan);
+cudaError_t fused_prepare(int device, int dtype, int V, int max_batch, int pin_cluster, int pin_threads, FusedPlan *plan);
 cudaError_t launch_fused(const VerifyParams &p, int dtype, const FusedPlan &plan, cudaStream_t stream,
                          uint64_t *launches);
-// how many CTAs of the split kernel are co-resident, and how many of them should share a row pair so that
-// the rows in flight stay inside L2 (1: not worth splitting)
-cudaError_t split_prepare(int device, int dtype, int V, int *resident_ctas, int *group_size);
-// copies the drafter table, flagging and replacing entries that must not be dereferenced (metasd_streaming.cu)
-cudaError_t launch_sanitize_table(const void *const *table, int K, const void *target, uint32_t mask, const void **clean,
-                                  uint32_t *status, cudaStream_t stream);
 // small state kernels (metasd_streaming.cu)
-cudaError_t launch_select(const BanditState &st, int batch, int32_t *arm_out, cudaStream_t stream);
 cudaError_t launch_reset(const BanditState &st, int max_batch, int K, int tau, int variant, double gamma,
                          uint32_t sequence_base, const int32_t *seq_ids, int n, cudaStream_t stream);
+
+// Host-side check of a state blob's payload against what the kernels index with (metasd_api.cu).
+int validate_state_payload(const metasd_config &cfg, const void *payload);
 
 }  // namespace metasd

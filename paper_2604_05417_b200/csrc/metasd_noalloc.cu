@@ -8,9 +8,10 @@
 // is part of the library image: every GPU that loads the library holds it until the process exits.
 //
 // The round it runs is the stateless part of metasd_verify: softmax statistics, accept tests, first
-// rejection, correction/bonus draw and the reward, launched as the same two streaming kernels.  There
-// is no bandit here (nothing persists between calls); the caller passes the round counter that keys
-// the random numbers.
+// rejection, correction/bonus draw and the reward, launched as the two streaming kernels a context
+// with the default configuration launches for the same logit type (the staged row-statistics kernel
+// for 16-byte aligned rows, the plain-load one otherwise, then the epilogue).  There is no bandit here
+// (nothing persists between calls); the caller passes the round counter that keys the random numbers.
 #include <mutex>
 
 #include "metasd_internal.h"
@@ -57,6 +58,8 @@ __global__ void noalloc_prepare_kernel(int batch, int32_t round)
 constexpr int MAX_DEVICES = 64;
 std::mutex g_setup_lock;
 StaticScratch *g_scratch_ptr[MAX_DEVICES];   // device address of the array on each device, once known
+RowGeometry g_geometry[MAX_DEVICES][2];      // launch shape of the row-statistics kernel per device and logit type
+bool g_geometry_ready[MAX_DEVICES][2];
 
 // Once per device, with that device current: ask the runtime where the array lives there.
 cudaError_t scratch_address(int device, StaticScratch **out)
@@ -69,6 +72,22 @@ cudaError_t scratch_address(int device, StaticScratch **out)
         g_scratch_ptr[device] = static_cast<StaticScratch *>(ptr);
     }
     *out = g_scratch_ptr[device];
+    return cudaSuccess;
+}
+
+// Once per device and logit type: the default launch shape and the function attribute (a larger dynamic
+// shared-memory window) its kernel needs.  Neither allocates device memory.
+cudaError_t default_geometry(int device, int dtype, RowGeometry *out)
+{
+    std::lock_guard<std::mutex> guard(g_setup_lock);
+    if (!g_geometry_ready[device][dtype]) {
+        metasd_config cfg;
+        metasd_default_config(&cfg);
+        cudaError_t e = streaming_prepare(device, dtype, cfg, &g_geometry[device][dtype]);
+        if (e != cudaSuccess) return e;
+        g_geometry_ready[device][dtype] = true;
+    }
+    *out = g_geometry[device][dtype];
     return cudaSuccess;
 }
 
@@ -96,6 +115,8 @@ extern "C" int metasd_verify_noalloc(int32_t batch, int32_t k, int32_t vocab, in
     if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= MAX_DEVICES) return METASD_ERR_CUDA;
     StaticScratch *scratch = nullptr;
     if (scratch_address(device, &scratch) != cudaSuccess) return METASD_ERR_CUDA;
+    RowGeometry geo;
+    if (default_geometry(device, logit_dtype, &geo) != cudaSuccess) return METASD_ERR_CUDA;
     cudaStream_t s = (cudaStream_t)stream;
 
     VerifyParams p = {};
@@ -115,11 +136,16 @@ extern "C" int metasd_verify_noalloc(int32_t batch, int32_t k, int32_t vocab, in
     p.status = &scratch->status;
     const size_t row_bytes = (size_t)vocab * (logit_dtype == METASD_BF16 ? 2 : 4);
     p.vector_ok = row_bytes % 16 == 0 && ((uintptr_t)target_logits % 16) == 0 && ((uintptr_t)draft_logits % 16) == 0;
+    {   // the share of every row that L2 is asked to keep between the sweeps: as in a default context
+        const long long nvec = (long long)row_bytes / 16;
+        p.keep_from_vec = (int32_t)(nvec - nvec * (logit_dtype == METASD_BF16 ? 750 : 900) / 1000);
+    }
+    p.poll_limit = 1u << 22;
 
     noalloc_prepare_kernel<<<(batch + 255) / 256, 256, 0, s>>>(batch, (int32_t)round);
     cudaError_t e = cudaGetLastError();
     uint64_t launches = 0;
-    if (e == cudaSuccess) e = launch_streaming(p, logit_dtype, s, &launches);
+    if (e == cudaSuccess) e = launch_streaming(p, logit_dtype, geo, s, &launches);
     if (e == cudaSuccess && status_out)
         e = cudaMemcpyAsync(status_out, &scratch->status, sizeof(uint32_t), cudaMemcpyDeviceToDevice, s);
     return e == cudaSuccess ? METASD_OK : METASD_ERR_CUDA;

@@ -4,29 +4,20 @@
 //                          row and the draft row with an online maximum, the target arg-max, then
 //                          sum_v min(p_v, q_v) = 1 - d_TV(p_j, q_j) (Definition 2) in a second
 //                          sweep over the same rows.  Writes one RowStats record.  Plain loads: any alignment.
-//   K1p row_stats_staged_kernel  K1 for 16-byte aligned rows (the default there): every thread stages its own
+//   K1p row_stats_staged_kernel  K1 for 16-byte aligned rows: every thread stages its own
 //                          vectors through shared memory with cp.async, several trips ahead, and the second
 //                          sweep starts on the trips that are still staged instead of reading them again.
-//   K1s split_row_stats_kernel  (opt-in) K1 with grp_size co-resident CTAs per row pair, each on its own part
-//                          of the vocabulary, exchanging (max, sum, arg-max) records through global memory.
+//   K1t row_stats_bulk_kernel    (metasd_bulk.cu) the same two sweeps by persistent CTAs whose rows arrive as TMA
+//                          bulk copies issued by one warp into a shared-memory ring.
 //   K2  epilogue_kernel    one CTA per sequence: accept tests with the Philox uniforms (Algorithm 4,
 //                          accept step), first rejection, inverse-CDF draw of the correction token from
 //                          max(0, p - q) or of the bonus token from p (its resampling step), the reward, the
 //                          bandit update and the next round's arm (Algorithm 2, update and selection steps).
-#include <stdlib.h>
-
 #include "metasd_device.cuh"
 
 namespace metasd {
 
 constexpr int K1_THREADS = 512;
-
-template <typename LT>
-__device__ __forceinline__ const LT *draft_rows(const VerifyParams &p, int b)
-{
-    if (p.draft) return reinterpret_cast<const LT *>(p.draft);
-    return reinterpret_cast<const LT *>(p.drafter_ptrs[p.st.arm[b]]);   // the table was checked by sanitize_table_kernel
-}
 
 // -------------------------------------------------------------------------------------------
 // K1
@@ -36,6 +27,7 @@ __global__ void __launch_bounds__(K1_THREADS) row_stats_kernel(const VerifyParam
 {
     constexpr int VEC = VECTOR ? Logit<LT>::VEC : 1;
     constexpr int NWARP = K1_THREADS / 32;
+    launch_dependents();   // the epilogue may be set up while this kernel runs; it waits for the whole grid before it reads
     const int j = blockIdx.x, b = blockIdx.y;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int V = p.V;
@@ -177,12 +169,6 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, uint64
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
-__device__ __forceinline__ uint4 lds16(uint32_t addr)
-{
-    uint4 v;
-    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
-    return v;
-}
 
 template <typename LT, int D, int THREADS, int MINB, bool BONUS_LAST>
 __global__ void __launch_bounds__(THREADS, MINB) row_stats_staged_kernel(const VerifyParams p)
@@ -192,6 +178,7 @@ __global__ void __launch_bounds__(THREADS, MINB) row_stats_staged_kernel(const V
     constexpr int NWARP = THREADS / 32;
     constexpr uint32_t ROW_STRIDE = THREADS * 16, STAGE_STRIDE = 2 * ROW_STRIDE;
     extern __shared__ __align__(16) unsigned char stage_mem[];   // [D][2 rows][THREADS] 16-byte slots
+    launch_dependents();   // the epilogue may be set up while this kernel runs; it waits for the whole grid before it reads
     // Blocks are dispatched in index order.  BONUS_LAST: the row pairs come first and the bonus rows (one row, half
     // the work) last, so that the launch ends on its shortest items (measured: better for the bf16 geometry, worse
     // for the fp32 one, which keeps the bonus rows interleaved).
@@ -410,229 +397,9 @@ __global__ void __launch_bounds__(THREADS, MINB) row_stats_staged_kernel(const V
 template <typename LT, int D, int THREADS, int MINB, bool BONUS_LAST>
 static cudaError_t launch_staged(const VerifyParams &p, dim3 grid, cudaStream_t stream)
 {
-    const size_t smem = (size_t)D * 2 * THREADS * 16;
-    cudaError_t e = cudaFuncSetAttribute(row_stats_staged_kernel<LT, D, THREADS, MINB, BONUS_LAST>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return e;
+    const size_t smem = (size_t)D * 2 * THREADS * 16;   // the attribute that allows it was set by streaming_prepare
     row_stats_staged_kernel<LT, D, THREADS, MINB, BONUS_LAST><<<grid, THREADS, smem, stream>>>(p);
     return cudaSuccess;
-}
-
-// -------------------------------------------------------------------------------------------
-// K1s
-// -------------------------------------------------------------------------------------------
-constexpr int KS_THREADS = 512;
-constexpr uint32_t KS_SPIN_LIMIT = 1u << 22;   // polls of 64 ns: a quarter of a second
-
-// Adds 1 without waiting for the result; the thread's earlier writes are visible to whoever sees the new count.
-__device__ __forceinline__ void red_release_inc(uint32_t *p)
-{
-    asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p) : "memory");
-}
-__device__ __forceinline__ uint32_t ld_acquire(const uint32_t *p)
-{
-    uint32_t v;
-    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-    return v;
-}
-
-// Warp 0 of every CTA only communicates: it publishes the CTA's record of a row pair (a release increment, no
-// round trip), waits (bounded) for the group's records, merges them for the second sweep, and afterwards
-// publishes the CTA's partial sum of min(p, q); the CTAs of a group take turns in adding the parts up.
-template <typename LT>
-__global__ void __launch_bounds__(KS_THREADS, 3) split_row_stats_kernel(const VerifyParams p)
-{
-    constexpr int VEC = Logit<LT>::VEC;
-    constexpr int NWARP = KS_THREADS / 32;          // warp 0 + NWARP - 1 sweeping warps
-    constexpr int NSWEEP = KS_THREADS - 32;         // sweeping threads
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int st = tid - 32;                        // index among the sweeping threads
-    const int V = p.V, G = p.grp_size;
-    const float c = p.c;
-    const int n_groups = gridDim.x / G, grp = blockIdx.x / G, g = blockIdx.x - grp * G;
-    const int nvec = V / VEC, per = (nvec + G - 1) / G;
-    const int v_lo = min(g * per, nvec), v_hi = min(v_lo + per, nvec);   // this CTA's part of every row
-    const uint64_t keep = l2_policy_evict_last(), drop = l2_policy_evict_first();
-    const int keep_from = v_hi - (int)((long long)(v_hi - v_lo) * p.keep_permille / 1000);
-    __shared__ MaxSum sh_a[NWARP], sh_b[NWARP];
-    __shared__ ArgMax sh_am[NWARP];
-    __shared__ double sh_min[NWARP];
-    __shared__ float sh_bcast[5];      // merged statistics of the row pair in its second sweep
-    __shared__ int sh_arg;
-    const int n_items = p.batch * (p.k + 1);
-
-    auto row_ptrs = [&](int item, const LT *&a, const LT *&d, bool &pair) {
-        const int b = item / (p.k + 1), j = item - b * (p.k + 1);
-        pair = j < p.k;
-        a = reinterpret_cast<const LT *>(p.target) + ((size_t)b * (p.k + 1) + j) * V;
-        d = pair ? draft_rows<LT>(p, b) + ((size_t)b * p.k + j) * V : nullptr;
-    };
-    // ---- sweeping warps: online (max, sum) of both rows, arg-max of the target row, over this CTA's part
-    auto first_sweep = [&](int item) {
-        const LT *a, *d;
-        bool pair;
-        row_ptrs(item, a, d, pair);
-        MaxSum sa = {METASD_NEG_BIG, 0.f}, sb = {METASD_NEG_BIG, 0.f};
-        ArgMax am = {METASD_NEG_BIG, 0x7FFFFFFF};
-        for (int i = v_lo + st; i < v_hi; i += NSWEEP) {
-            float xa[VEC], xb[VEC];
-            // the end of this CTA's part is asked to stay in L2 until the second sweep (which starts there)
-            const uint64_t pol = i >= keep_from ? keep : drop;
-            Logit<LT>::unpack(ld_stream_hint(reinterpret_cast<const uint4 *>(a) + i, pol), xa);
-            if (pair) Logit<LT>::unpack(ld_stream_hint(reinterpret_cast<const uint4 *>(d) + i, pol), xb);
-            float cm = xa[0];
-#pragma unroll
-            for (int e = 1; e < VEC; ++e) cm = fmaxf(cm, xa[e]);
-            if (cm > sa.m) {
-                sa.s *= ex2((sa.m - cm) * c);
-                sa.m = cm;
-                int first = 0;
-#pragma unroll
-                for (int e = VEC - 1; e >= 0; --e)
-                    if (xa[e] == cm) first = e;
-                am.v = cm;
-                am.i = i * VEC + first;
-            }
-            const float nma = -sa.m * c;
-#pragma unroll
-            for (int e = 0; e < VEC; ++e) sa.s += ex2(fmaf(xa[e], c, nma));
-            if (pair) {
-                float bm = xb[0];
-#pragma unroll
-                for (int e = 1; e < VEC; ++e) bm = fmaxf(bm, xb[e]);
-                if (bm > sb.m) {
-                    sb.s *= ex2((sb.m - bm) * c);
-                    sb.m = bm;
-                }
-                const float nmb = -sb.m * c;
-#pragma unroll
-                for (int e = 0; e < VEC; ++e) sb.s += ex2(fmaf(xb[e], c, nmb));
-            }
-        }
-        sa = warp_merge(sa, c);
-        sb = warp_merge(sb, c);
-        am = warp_argmax(am);
-        if (lane == 0) { sh_a[warp] = sa; sh_b[warp] = sb; sh_am[warp] = am; }
-    };
-    // ---- sweeping warps: sum_v min(p_v, q_v) = (1 / sum_a) sum_v 2^min(ya_v, yb_v) over this CTA's part
-    auto second_sweep = [&](int item) {
-        const LT *a, *d;
-        bool pair;
-        row_ptrs(item, a, d, pair);
-        double w = 0.0;
-        if (pair) {
-            const float nma = -sh_bcast[0] * c, nmb = sh_bcast[4], sum_a = sh_bcast[1];
-            float acc = 0.f;
-            for (int i = v_hi - 1 - st; i >= v_lo; i -= NSWEEP) {   // backwards: the end was read last
-                float xa[VEC], xb[VEC];
-                Logit<LT>::unpack(ld_stream_hint(reinterpret_cast<const uint4 *>(a) + i, drop), xa);
-                Logit<LT>::unpack(ld_stream_hint(reinterpret_cast<const uint4 *>(d) + i, drop), xb);
-#pragma unroll
-                for (int e = 0; e < VEC; ++e) acc += ex2(fminf(fmaf(xa[e], c, nma), fmaf(xb[e], c, nmb)));
-            }
-            w = warp_sum((double)(acc / sum_a));
-        }
-        if (lane == 0) sh_min[warp] = w;
-    };
-    // ---- warp 0: the CTA's record of a first sweep goes to global memory
-    auto publish_record = [&](int item) {
-        MaxSum ra = (lane >= 1 && lane < NWARP) ? sh_a[lane] : MaxSum{METASD_NEG_BIG, 0.f};
-        MaxSum rb = (lane >= 1 && lane < NWARP) ? sh_b[lane] : MaxSum{METASD_NEG_BIG, 0.f};
-        ArgMax rm = (lane >= 1 && lane < NWARP) ? sh_am[lane] : ArgMax{METASD_NEG_BIG, 0x7FFFFFFF};
-        ra = warp_merge(ra, c);
-        rb = warp_merge(rb, c);
-        rm = warp_argmax(rm);
-        if (lane == 0) {
-            GroupRecord r;
-            r.max_a = ra.m; r.sum_a = ra.s; r.max_b = rb.m; r.sum_b = rb.s; r.argmax_a = rm.i;
-            r.pad[0] = r.pad[1] = r.pad[2] = 0;
-            p.grp_rec[(size_t)item * G + g] = r;
-            red_release_inc(&p.grp_count[item]);
-        }
-    };
-    // ---- warp 0: wait (bounded) for the group's records of a row pair and merge them for its second sweep
-    auto merge_group = [&](int item) {
-        if (lane == 0) {
-            uint32_t it = 0;
-            while (ld_acquire(&p.grp_count[item]) < (uint32_t)G) {
-                if (++it > KS_SPIN_LIMIT) { atomicOr(p.status, METASD_STATUS_TIMEOUT); break; }
-                __nanosleep(64);
-            }
-        }
-        __syncwarp();
-        MaxSum ga = {METASD_NEG_BIG, 0.f}, gb = {METASD_NEG_BIG, 0.f};
-        ArgMax gm = {METASD_NEG_BIG, 0x7FFFFFFF};
-        if (lane < G) {
-            const int4 *src = reinterpret_cast<const int4 *>(p.grp_rec + (size_t)item * G + lane);
-            const int4 lo = __ldcg(src), hi = __ldcg(src + 1);
-            ga.m = __int_as_float(lo.x); ga.s = __int_as_float(lo.y);
-            gb.m = __int_as_float(lo.z); gb.s = __int_as_float(lo.w);
-            gm.v = ga.m; gm.i = hi.x;
-        }
-        ga = warp_merge(ga, c);
-        gb = warp_merge(gb, c);
-        gm = warp_argmax(gm);
-        if (lane == 0) {
-            sh_bcast[0] = ga.m; sh_bcast[1] = ga.s; sh_bcast[2] = gb.m; sh_bcast[3] = gb.s;
-            // q_v / p_v = 2^(yb - ya) sum_a / sum_b: the ratio of the sums folds into the draft row's offset
-            sh_bcast[4] = -gb.m * c + log2f(ga.s / gb.s);
-            sh_arg = gm.i;
-        }
-    };
-    // ---- warp 0: this CTA's part of sum min(p, q)
-    auto publish_min = [&](int item) {
-        if (lane == 0) {
-            double part = 0.0;
-            for (int i = 1; i < NWARP; ++i) part += sh_min[i];
-            p.grp_min[(size_t)item * G + g] = part;
-            red_release_inc(&p.grp_count[item]);
-        }
-    };
-    // ---- warp 0 of one CTA of the group (they take turns): once every part is in, add the parts up and write the
-    //      row pair's statistics
-    auto finalise = [&](int item, float max_a, float sum_a, float max_b, float sum_b, int arg) {
-        if (lane == 0) {
-            uint32_t it = 0;
-            while (ld_acquire(&p.grp_count[item]) < 2u * (uint32_t)G) {
-                if (++it > KS_SPIN_LIMIT) { atomicOr(p.status, METASD_STATUS_TIMEOUT); break; }
-                __nanosleep(64);
-            }
-            const bool pair = item % (p.k + 1) < p.k;
-            double total = 0.0;
-            for (int i = 0; i < G; ++i) total += __ldcg(p.grp_min + (size_t)item * G + i);
-            RowStats r;
-            r.max_a = max_a; r.sum_a = sum_a; r.max_b = max_b; r.sum_b = sum_b;
-            r.argmax_a = arg;
-            uint32_t flags = 0;
-            // NaN or +Inf anywhere makes the sum NaN; an all -Inf row leaves it 0
-            const bool bad_a = !(sum_a > 0.f) || !(sum_a < INFINITY) || !(max_a < INFINITY);
-            const bool bad_b = pair && (!(sum_b > 0.f) || !(sum_b < INFINITY) || !(max_b < INFINITY));
-            if (bad_a || bad_b) flags |= METASD_STATUS_NONFINITE;
-            r.sum_min = flags ? 0.0 : total;
-            r.flags = flags;
-            p.stats[item] = r;
-        }
-    };
-
-    // Group grp takes row pairs grp, grp + n_groups, ... in (sequence, position) order: both sweeps of a row pair
-    // back to back (the second finds the first's bytes in L2), the group's exchange in between.
-    float m_a = 0.f, s_a = 0.f, m_b = 0.f, s_b = 0.f;
-    int arg = 0, turn = 0;
-    for (int item = grp; item < n_items; item += n_groups, ++turn) {
-        if (warp != 0) first_sweep(item);
-        __syncthreads();
-        if (warp == 0) {
-            publish_record(item);
-            merge_group(item);
-            m_a = sh_bcast[0]; s_a = sh_bcast[1]; m_b = sh_bcast[2]; s_b = sh_bcast[3]; arg = sh_arg;
-        }
-        __syncthreads();
-        if (warp != 0) second_sweep(item);
-        __syncthreads();
-        if (warp == 0) {
-            publish_min(item);
-            if (turn % G == g) finalise(item, m_a, s_a, m_b, s_b, arg);   // the CTAs of a group take turns
-        }
-    }
 }
 
 // -------------------------------------------------------------------------------------------
@@ -774,51 +541,45 @@ __device__ __forceinline__ int warp_find_part(const double *x, int n, double bas
     return part;
 }
 
-// Inverse CDF in token order over one row (pair): the smallest v with sum_{w<=v} weight_w > u * total.
-// Every warp owns a contiguous range of vectors; totals and offsets are carried in fp64.
-template <typename LT, bool VECTOR, int K2_THREADS>
-__device__ int block_inverse_cdf(const LT *a, const LT *d, int V, int mode, float u, float c, float max_a,
-                                 float sum_a, float max_b, float sum_b, double *sh_tot, double *sh_sub, int *sh_tok)
-{
-    constexpr int VEC = VECTOR ? Logit<LT>::VEC : 1;
-    constexpr int NWARP = K2_THREADS / 32;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int nvec = V / VEC;
-    const int per_warp = (nvec + NWARP - 1) / NWARP;
-    const int v0 = min(warp * per_warp, nvec), v1 = min(v0 + per_warp, nvec);
-    const float nma = -max_a * c, nmb = -max_b * c;
-    const float ia = 1.0f / sum_a, ib = 1.0f / sum_b;
+// Shared-memory work space of the draw.
+constexpr int DRAW_MAX_SEG = 64;
+template <int NWARP> struct DrawShared {
+    double tot[2][NWARP];            // warp totals of a segment, double-buffered by segment parity
+    double sub[NWARP];               // warp totals of the second search level
+    double seg[DRAW_MAX_SEG];        // weight of every segment walked so far
+    double before;                   // weight in front of the token that was found
+    int tok;
+};
 
-    const double acc = warp_range_sum<LT, VEC>(a, d, v0, v1, mode, c, nma, ia, nmb, ib);
-    if (lane == 0) sh_tot[warp] = acc;
-    if (tid == 0) *sh_tok = -1;
-    __syncthreads();
-    // the warp whose range holds the crossing; rounding may leave none: then the last warp with mass
-    double threshold = (double)u, base, total;
-    const int wstar = warp_find_part<true>(sh_tot, NWARP, 0.0, threshold, base, total);
-    if (!(total > 0.0)) { __syncthreads(); return -1; }
-    // second level: each warp takes a part of that range, so that the final scan is a trip or two instead of a
-    // long chain of dependent loads in one warp
-    const int r0 = min(wstar * per_warp, nvec), r1 = min(r0 + per_warp, nvec);
+// Second search level: the smallest token v in the vectors [r0, r1) with base + sum_{w in range, w <= v} weight_w >
+// threshold; rounding may leave none, then the last token of the range with mass (-1 if it has none).  Every warp
+// sums a part of the range, one warp-parallel scan finds the part that holds the crossing and the owning warp
+// finishes with a lane scan.  `before` receives base + the weight in front of the token.  The whole CTA takes part.
+template <typename LT, int VEC, int NWARP>
+__device__ int locate_in_range(const LT *a, const LT *d, int r0, int r1, int mode, float c, float nma, float ia, float nmb,
+                               float ib, double base, double threshold, DrawShared<NWARP> &sh, double &before)
+{
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int per_sub = (r1 - r0 + NWARP - 1) / NWARP;
     const int s0 = min(r0 + warp * per_sub, r1), s1 = min(s0 + per_sub, r1);
     {
         const double acc2 = warp_range_sum<LT, VEC>(a, d, s0, s1, mode, c, nma, ia, nmb, ib);
-        if (lane == 0) sh_sub[warp] = acc2;
+        if (lane == 0) sh.sub[warp] = acc2;
+        if (tid == 0) { sh.tok = -1; sh.before = base; }
     }
     __syncthreads();
-    double total2;
-    const int sstar = warp_find_part<false>(sh_sub, NWARP, base, threshold, base, total2);
+    double total2, sub_base;
+    const int sstar = warp_find_part<false>(sh.sub, NWARP, base, threshold, sub_base, total2);
     if (warp == sstar) {
-        const int v0 = s0, v1 = s1;
         int found = -1, last_pos = -1;
-        double run_base = base;
-        for (int i0 = v0; i0 < v1 && found < 0; i0 += 32) {
+        double found_before = sub_base, last_before = sub_base;
+        double run_base = sub_base;
+        for (int i0 = s0; i0 < s1 && found < 0; i0 += 32) {
             const int i = i0 + lane;
             float w[VEC];
 #pragma unroll
             for (int e = 0; e < VEC; ++e) w[e] = 0.f;
-            if (i < v1) draw_weights<LT, VEC>(a, d, i, mode, c, nma, ia, nmb, ib, w);
+            if (i < s1) draw_weights<LT, VEC>(a, d, i, mode, c, nma, ia, nmb, ib, w);
             float s = 0.f;
 #pragma unroll
             for (int e = 0; e < VEC; ++e) s += w[e];
@@ -830,9 +591,14 @@ __device__ int block_inverse_cdf(const LT *a, const LT *d, int V, int mode, floa
             }
             const bool crosses = run_base + incl > threshold;
             const unsigned ballot = __ballot_sync(0xFFFFFFFFu, crosses);
+            {
+                double cum = run_base + incl - (double)s;
 #pragma unroll
-            for (int e = 0; e < VEC; ++e)
-                if (w[e] > 0.f) last_pos = i * VEC + e;
+                for (int e = 0; e < VEC; ++e) {
+                    if (w[e] > 0.f) { last_pos = i * VEC + e; last_before = cum; }
+                    cum += (double)w[e];
+                }
+            }
             if (ballot) {
                 const int src = __ffs(ballot) - 1;
                 if (lane == src) {
@@ -840,31 +606,113 @@ __device__ int block_inverse_cdf(const LT *a, const LT *d, int V, int mode, floa
                     int tok = -1;
 #pragma unroll
                     for (int e = 0; e < VEC; ++e) {
+                        if (tok < 0 && cum + (double)w[e] > threshold) { tok = i * VEC + e; found_before = cum; }
                         cum += (double)w[e];
-                        if (tok < 0 && cum > threshold) tok = i * VEC + e;
                     }
                     // the vector's own sum crossed, so an element does unless rounding interferes
-                    if (tok < 0) {
-#pragma unroll
-                        for (int e = 0; e < VEC; ++e)
-                            if (w[e] > 0.f) tok = i * VEC + e;
-                    }
+                    if (tok < 0) { tok = last_pos; found_before = last_before; }
                     found = tok;
                 }
                 found = __shfl_sync(0xFFFFFFFFu, found, src);
+                found_before = __shfl_sync(0xFFFFFFFFu, found_before, src);
             }
             run_base += __shfl_sync(0xFFFFFFFFu, incl, 31);
         }
-        if (found < 0) {  // rounding left the running sum a hair under the threshold
+        if (found < 0) {  // rounding left the running sum a hair under the threshold: the last token with mass
+            int best = last_pos;
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) last_pos = max(last_pos, __shfl_xor_sync(0xFFFFFFFFu, last_pos, o));
-            found = last_pos;
+            for (int o = 16; o > 0; o >>= 1) best = max(best, __shfl_xor_sync(0xFFFFFFFFu, best, o));
+            const unsigned who = __ballot_sync(0xFFFFFFFFu, best >= 0 && last_pos == best);
+            found = best;
+            if (who) found_before = __shfl_sync(0xFFFFFFFFu, last_before, __ffs(who) - 1);
         }
-        if (lane == 0) *sh_tok = found;
+        if (lane == 0) { sh.tok = found; sh.before = found_before; }
     }
     __syncthreads();
-    return *sh_tok;
+    before = sh.before;
+    return sh.tok;
 }
+
+// Inverse CDF in token order over one row (pair): the smallest v with sum_{w<=v} weight_w > u * total, where total is
+// the sum of all the weights as this walk adds them up (fp32 weights, fp64 sums).  The walk goes through the row in
+// token order, one segment at a time with the whole CTA on the segment, and stops behind the segment that holds the
+// crossing: `approx_total` is the total as the row statistics already give it (1 - sum_v min(p_v, q_v) for the
+// residual, 1 for the bonus row), equal to the walk's own total to within `guard`.  A token is taken early only if
+// it is the answer for every total in approx_total +- guard; otherwise (a CDF edge inside that band, or a total too
+// small for the band to mean anything) the walk goes on to the end of the row and decides with its own total.  The
+// answer is therefore always the one of the full walk.  Returns -1 when the row has no mass.
+template <typename LT, bool VECTOR, int K2_THREADS>
+__device__ int block_inverse_cdf(const LT *a, const LT *d, int V, int mode, float u, float c, float max_a, float sum_a,
+                                 float max_b, float sum_b, double approx_total, DrawShared<K2_THREADS / 32> &sh)
+{
+    constexpr int VEC = VECTOR ? Logit<LT>::VEC : 1;
+    constexpr int NWARP = K2_THREADS / 32;
+    constexpr double guard = 2.0e-5;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int nvec = V / VEC;
+    const float nma = -max_a * c, nmb = -max_b * c;
+    const float ia = 1.0f / sum_a, ib = 1.0f / sum_b;
+    // segments of at least 128 vectors per warp (four 16-byte loads per lane in flight), at most DRAW_MAX_SEG of them
+    int per_warp = 128;
+    {
+        const long long need = ((long long)nvec + DRAW_MAX_SEG - 1) / DRAW_MAX_SEG;
+        const int pw = (int)((need + NWARP - 1) / NWARP);
+        if (pw > per_warp) per_warp = (pw + 31) & ~31;
+    }
+    const int seg_vecs = per_warp * NWARP;
+    const int n_seg = (nvec + seg_vecs - 1) / seg_vecs;
+    const bool early = approx_total > 16.0 * guard;
+    const double lo = (double)u * (approx_total - guard), hi = (double)u * (approx_total + guard);
+
+    double running = 0.0, seg_start = 0.0;
+    int s = 0, stop = -1;
+    for (; s < n_seg; ++s) {
+        const int g0 = s * seg_vecs;
+        const int v0 = min(g0 + warp * per_warp, nvec), v1 = min(v0 + per_warp, nvec);
+        const double acc = warp_range_sum<LT, VEC>(a, d, v0, v1, mode, c, nma, ia, nmb, ib);
+        if (lane == 0) sh.tot[s & 1][warp] = acc;
+        __syncthreads();
+        // every warp adds the warps' totals up in the same order
+        double x0 = lane < NWARP ? sh.tot[s & 1][lane] : 0.0;
+        if (NWARP > 32) x0 += lane + 32 < NWARP ? sh.tot[s & 1][lane + 32] : 0.0;
+        const double seg_total = warp_sum(x0);
+        if (tid == 0) sh.seg[s] = seg_total;
+        seg_start = running;
+        running += seg_total;
+        if (early && stop < 0 && running > hi) { stop = s; ++s; break; }
+    }
+    if (stop >= 0 && seg_start <= lo) {
+        // for every total in the band the crossing lies in segment `stop`: find it for the upper end of the band and
+        // take it if the weight in front of it does not reach the lower end
+        const int r0 = stop * seg_vecs, r1 = min(r0 + seg_vecs, nvec);
+        double before;
+        const int tok = locate_in_range<LT, VEC, NWARP>(a, d, r0, r1, mode, c, nma, ia, nmb, ib, seg_start, hi, sh, before);
+        if (tok >= 0 && before <= lo) return tok;
+    }
+    // the band did not decide: the rest of the row, then the walk's own total
+    for (; s < n_seg; ++s) {
+        const int g0 = s * seg_vecs;
+        const int v0 = min(g0 + warp * per_warp, nvec), v1 = min(v0 + per_warp, nvec);
+        const double acc = warp_range_sum<LT, VEC>(a, d, v0, v1, mode, c, nma, ia, nmb, ib);
+        if (lane == 0) sh.tot[s & 1][warp] = acc;
+        __syncthreads();
+        double x0 = lane < NWARP ? sh.tot[s & 1][lane] : 0.0;
+        if (NWARP > 32) x0 += lane + 32 < NWARP ? sh.tot[s & 1][lane + 32] : 0.0;
+        const double seg_total = warp_sum(x0);
+        if (tid == 0) sh.seg[s] = seg_total;
+    }
+    __syncthreads();
+    double threshold = (double)u, base, total;
+    const int sstar = warp_find_part<true>(sh.seg, n_seg, 0.0, threshold, base, total);
+    if (!(total > 0.0)) { __syncthreads(); return -1; }
+    const int r0 = min(sstar * seg_vecs, nvec), r1 = min(r0 + seg_vecs, nvec);
+    double before;
+    return locate_in_range<LT, VEC, NWARP>(a, d, r0, r1, mode, c, nma, ia, nmb, ib, base, threshold, sh, before);
+}
+
+// Blocks until the kernel launched before this one in the stream has finished and its writes are visible (a no-op
+// when this kernel was launched without programmatic stream serialisation).
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 // K2_THREADS: the draw walks one row pair per sequence, so a small batch wants large CTAs (many warps keep the
 // load chains short) and a large batch wants many small ones.
@@ -873,22 +721,32 @@ __global__ void __launch_bounds__(K2_THREADS, 1024 / K2_THREADS) epilogue_kernel
 {
     const int b = blockIdx.x, tid = threadIdx.x;
     const int k_slots = p.k, V = p.V, K = p.K;   // rows and tokens are laid out for k_slots positions per sequence
-    const int k = drafted(p.draft_len, b, k_slots);   // positions this sequence drafted this round
     const float c = p.c;
-    const LT *target = reinterpret_cast<const LT *>(p.target) + (size_t)b * (k_slots + 1) * V;
-    const LT *draft = draft_rows<LT>(p, b) + (size_t)b * k_slots * V;
-    const RowStats *stats = p.stats + (size_t)b * (k_slots + 1);
 
     __shared__ int sh_nacc, sh_mode, sh_tok;
     __shared__ float sh_u;
     __shared__ uint32_t sh_flags;
     __shared__ double sh_reward;
-    __shared__ double sh_tot[K2_THREADS / 32], sh_sub[K2_THREADS / 32];   // warp totals of the two search levels
+    __shared__ DrawShared<K2_THREADS / 32> sh_draw;
     __shared__ int sh_accept[16];
     __shared__ double sh_align[16];
 
+    // The row-statistics kernel may still be running when this kernel starts (programmatic stream serialisation):
+    // nothing it writes is read, and nothing it reads is written, before this wait.
+    grid_dependency_wait();
+
+    const int k = drafted(p.draft_len, b, k_slots);   // positions this sequence drafted this round
+    const LT *target = reinterpret_cast<const LT *>(p.target) + (size_t)b * (k_slots + 1) * V;
+    const LT *draft = draft_rows<LT>(p, b) + (size_t)b * k_slots * V;
+    const RowStats *stats = p.stats + (size_t)b * (k_slots + 1);
+
     if (tid == 0) sh_flags = (p.draft_len && p.draft_len[b] != k) ? METASD_STATUS_BAD_LENGTH : 0u;
     __syncthreads();
+    // pointer-table mode: an entry that must not be dereferenced is flagged once per call, played or not
+    if (b == 0 && p.drafter_ptrs && tid < K) {
+        const void *q = p.drafter_ptrs[tid];
+        if (q == nullptr || (reinterpret_cast<uintptr_t>(q) & p.table_mask) != 0) atomicOr(&sh_flags, METASD_STATUS_BAD_POINTER);
+    }
     const int t = p.st.t[b];
     const int arm = p.st.arm[b];
     if (tid < k) {
@@ -931,7 +789,7 @@ __global__ void __launch_bounds__(K2_THREADS, 1024 / K2_THREADS) epilogue_kernel
     }
     __syncthreads();
     if (tid == 0) {
-        // first rejection (Algorithm 4, "exit for loop"), reward (Definition 2), what to draw
+        // first rejection (Algorithm 4, the rejection step ends the loop), reward (Definition 2), what to draw
         int n_acc = k;
         double sum_align = 0.0;
         for (int j = k - 1; j >= 0; --j)
@@ -957,17 +815,18 @@ __global__ void __launch_bounds__(K2_THREADS, 1024 / K2_THREADS) epilogue_kernel
 
     int token = sh_tok;
     const int mode = sh_mode, n_acc = sh_nacc;
-    __syncthreads();
     if (mode != 0) {
         const RowStats rs = stats[n_acc];
         const LT *a = target + (size_t)n_acc * V;
         const LT *d = mode == 1 ? draft + (size_t)n_acc * V : nullptr;
+        // the total of the draw's weights as the row statistics give it: sum max(0, p - q) = 1 - sum min(p, q); sum p = 1
+        const double known = mode == 1 ? 1.0 - rs.sum_min : 1.0;
         token = block_inverse_cdf<LT, VECTOR, K2_THREADS>(a, d, V, mode, sh_u, c, rs.max_a, rs.sum_a, rs.max_b, rs.sum_b,
-                                              sh_tot, sh_sub, &sh_tok);
+                                                          known, sh_draw);
         if (token < 0 && mode == 1) {  // p == q in fp32 yet rejected: draw from p
-            __syncthreads();   // every thread has read the first draw's answer before the slot is reused
+            __syncthreads();   // every thread has read the first draw's answer before the work space is reused
             token = block_inverse_cdf<LT, VECTOR, K2_THREADS>(a, nullptr, V, 2, sh_u, c, rs.max_a, rs.sum_a, rs.max_b,
-                                                  rs.sum_b, sh_tot, sh_sub, &sh_tok);
+                                                              rs.sum_b, 1.0, sh_draw);
         }
     }
 
@@ -989,123 +848,113 @@ __global__ void __launch_bounds__(K2_THREADS, 1024 / K2_THREADS) epilogue_kernel
 // -------------------------------------------------------------------------------------------
 // launchers
 // -------------------------------------------------------------------------------------------
-template <typename LT>
-static cudaError_t launch_streaming_t(const VerifyParams &p, cudaStream_t stream, uint64_t *launches)
+// The built shapes of the staged kernel, per logit type: (threads, stages, CTAs per SM, bonus rows last).
+#define METASD_STAGED_SHAPES(X) X(512, 4, 3, true) X(1024, 6, 1, false) X(1024, 4, 1, true) X(768, 6, 2, true) X(384, 4, 4, true)
+
+template <typename LT, int D, int THREADS, int MINB, bool BONUS_LAST>
+static cudaError_t prepare_staged()
 {
-    dim3 g1(p.k + 1, p.batch);
-    const bool big_ctas = p.batch <= 320;   // up to about two sequences per SM
-    if (p.vector_ok && p.grp_size > 1 && !p.draft_len) {
-        const int n_items = p.batch * (p.k + 1);
-        int n_groups = p.grp_ctas / p.grp_size;
-        if (n_groups > n_items) n_groups = n_items;
-        cudaError_t e = cudaMemsetAsync(p.grp_count, 0, (size_t)n_items * sizeof(uint32_t), stream);
-        if (e != cudaSuccess) return e;
-        // the CTAs of a group wait on one another: a cooperative launch guarantees that they are co-resident
-        VerifyParams q = p;
-        void *args[] = {&q};
-        e = cudaLaunchCooperativeKernel(reinterpret_cast<const void *>(&split_row_stats_kernel<LT>), dim3(n_groups * p.grp_size),
-                                        dim3(KS_THREADS), args, 0, stream);
-        if (e != cudaSuccess) return e;
-    } else if (p.vector_ok && p.k1_stages > 1) {
-        // Measured on B200: bf16 rows (8 logits per 16 bytes) are bound by arithmetic as much as by memory: 3 x 512
-        // threads per SM (4 x 384 is as fast in short runs but moves 7 % more HBM bytes, which costs clock under
-        // the power cap); fp32 rows (4 logits per 16 bytes) are bound by memory and want few row pairs in flight
-        // and a large share of each kept in shared memory: 1 x 1024 threads per SM, 6 stages (192 KB).
-        cudaError_t e;
-        const dim3 gp((unsigned)p.batch * (unsigned)(p.k + 1));
-        if constexpr (sizeof(LT) == 2) e = launch_staged<LT, 4, 512, 3, true>(p, gp, stream);
-        else e = launch_staged<LT, 6, 1024, 1, false>(p, gp, stream);
-        if (e != cudaSuccess) return e;
-    } else if (p.vector_ok) {
-        row_stats_kernel<LT, true><<<g1, K1_THREADS, 0, stream>>>(p);
-    } else {
-        row_stats_kernel<LT, false><<<g1, K1_THREADS, 0, stream>>>(p);
+    return cudaFuncSetAttribute(row_stats_staged_kernel<LT, D, THREADS, MINB, BONUS_LAST>,
+                                cudaFuncAttributeMaxDynamicSharedMemorySize, D * 2 * THREADS * 16);
+}
+
+template <typename LT>
+static cudaError_t prepare_staged_t(int threads, int stages, int *per_sm)
+{
+#define X(T, D, M, BL) if (threads == T && stages == D) { *per_sm = M; return prepare_staged<LT, D, T, M, BL>(); }
+    METASD_STAGED_SHAPES(X)
+#undef X
+    return cudaErrorNotSupported;
+}
+
+template <typename LT>
+static cudaError_t launch_staged_t(const VerifyParams &p, const RowGeometry &geo, cudaStream_t stream)
+{
+    const dim3 grid((unsigned)p.batch * (unsigned)(p.k + 1));
+#define X(T, D, M, BL) if (geo.threads == T && geo.stages == D) return launch_staged<LT, D, T, M, BL>(p, grid, stream);
+    METASD_STAGED_SHAPES(X)
+#undef X
+    return cudaErrorNotSupported;
+}
+
+// Resolves the row-statistics shape for a context and sets the launch attributes its kernels need, once.
+// Measured on B200: bf16 rows (8 logits per 16 bytes) are bound by arithmetic as much as by memory, fp32 rows (4 logits
+// per 16 bytes) by memory: they want few row pairs in flight and a large share of each kept in shared memory.
+cudaError_t streaming_prepare(int device, int dtype, const metasd_config &cfg, RowGeometry *geo)
+{
+    cudaError_t e = cudaDeviceGetAttribute(&geo->n_sm, cudaDevAttrMultiProcessorCount, device);
+    if (e != cudaSuccess) return e;
+    geo->kernel = cfg.row_kernel == METASD_ROWS_AUTO ? METASD_ROWS_STAGED : cfg.row_kernel;
+    geo->threads = cfg.row_threads;
+    geo->stages = cfg.row_stages;
+    geo->per_sm = 1;
+    if (geo->kernel == METASD_ROWS_PLAIN) {
+        if (geo->threads && geo->threads != K1_THREADS) return cudaErrorNotSupported;
+        geo->threads = K1_THREADS;
+        geo->stages = 0;
+        geo->per_sm = 3;
+        return cudaSuccess;
     }
-    {
-        if (!p.vector_ok) {
-            if (big_ctas) epilogue_kernel<LT, false, 512><<<p.batch, 512, 0, stream>>>(p);
-            else epilogue_kernel<LT, false, 256><<<p.batch, 256, 0, stream>>>(p);
-        } else {
-            if (big_ctas) epilogue_kernel<LT, true, 512><<<p.batch, 512, 0, stream>>>(p);
-            else epilogue_kernel<LT, true, 256><<<p.batch, 256, 0, stream>>>(p);
-        }
+    if (geo->kernel == METASD_ROWS_BULK) {
+        if (!geo->threads) geo->threads = 1024;
+        if (!geo->stages) geo->stages = 6;
+        return bulk_prepare(dtype, geo);
+    }
+    if (geo->kernel != METASD_ROWS_STAGED) return cudaErrorNotSupported;
+    if (!geo->threads) geo->threads = dtype == METASD_BF16 ? 512 : 1024;
+    if (!geo->stages) geo->stages = dtype == METASD_BF16 ? 4 : 6;
+    return dtype == METASD_BF16 ? prepare_staged_t<__nv_bfloat16>(geo->threads, geo->stages, &geo->per_sm)
+                                : prepare_staged_t<float>(geo->threads, geo->stages, &geo->per_sm);
+}
+
+template <typename LT>
+static cudaError_t launch_streaming_t(const VerifyParams &p, const RowGeometry &geo, cudaStream_t stream, uint64_t *launches)
+{
+    cudaError_t e = cudaSuccess;
+    if (!p.vector_ok) {
+        row_stats_kernel<LT, false><<<dim3(p.k + 1, p.batch), K1_THREADS, 0, stream>>>(p);
+    } else if (geo.kernel == METASD_ROWS_BULK) {
+        e = launch_row_stats_bulk(p, sizeof(LT) == 2 ? METASD_BF16 : METASD_FP32, geo, stream);
+    } else if (geo.kernel == METASD_ROWS_STAGED) {
+        e = launch_staged_t<LT>(p, geo, stream);
+    } else {
+        row_stats_kernel<LT, true><<<dim3(p.k + 1, p.batch), K1_THREADS, 0, stream>>>(p);
+    }
+    if (e != cudaSuccess) return e;
+    if ((e = cudaGetLastError()) != cudaSuccess) return e;
+    // The epilogue is launched with programmatic stream serialisation: its blocks may be set up while the
+    // row-statistics kernel drains, and wait (griddepcontrol.wait) for its completion before they read anything.
+    const bool big_ctas = p.batch <= 320;   // up to about two sequences per SM
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)p.batch);
+    cfg.blockDim = dim3(big_ctas ? 512u : 256u);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute at;
+    at.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &at;
+    cfg.numAttrs = 1;
+    if (!p.vector_ok) {
+        if (big_ctas) e = cudaLaunchKernelEx(&cfg, epilogue_kernel<LT, false, 512>, p);
+        else e = cudaLaunchKernelEx(&cfg, epilogue_kernel<LT, false, 256>, p);
+    } else {
+        if (big_ctas) e = cudaLaunchKernelEx(&cfg, epilogue_kernel<LT, true, 512>, p);
+        else e = cudaLaunchKernelEx(&cfg, epilogue_kernel<LT, true, 256>, p);
     }
     *launches += 2;
-    return cudaGetLastError();
+    return e;
 }
 
-cudaError_t launch_streaming(const VerifyParams &p, int dtype, cudaStream_t stream, uint64_t *launches)
+cudaError_t launch_streaming(const VerifyParams &p, int dtype, const RowGeometry &geo, cudaStream_t stream, uint64_t *launches)
 {
-    if (dtype == METASD_BF16) return launch_streaming_t<__nv_bfloat16>(p, stream, launches);
-    return launch_streaming_t<float>(p, stream, launches);
-}
-
-cudaError_t split_prepare(int device, int dtype, int V, int *resident_ctas, int *group_size)
-{
-    *resident_ctas = 0;
-    *group_size = 1;
-    int per_sm = 0, n_sm = 0, l2 = 0, coop = 0;
-    cudaError_t e;
-    if (dtype == METASD_BF16)
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, split_row_stats_kernel<__nv_bfloat16>, KS_THREADS, 0);
-    else
-        e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, split_row_stats_kernel<float>, KS_THREADS, 0);
-    if (e != cudaSuccess) return e;
-    if ((e = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, device)) != cudaSuccess) return e;
-    if ((e = cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, device)) != cudaSuccess) return e;
-    if ((e = cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, device)) != cudaSuccess) return e;
-    if (!coop || per_sm < 1) return cudaSuccess;
-    const int resident = per_sm * n_sm;
-    // row-pair bytes in flight = resident CTAs x (row pair / group size); keep them within a third of L2
-    const double pair_bytes = 2.0 * V * (dtype == METASD_BF16 ? 2 : 4);
-    const char *pin = getenv("METASD_SPLIT_GROUP");
-    // measured on B200: the exchange costs more than the saved HBM traffic gains, so splitting is opt-in
-    // (METASD_SPLIT_GROUP); the L2-sized default would be ceil(resident * pair_bytes / (l2 / 3))
-    (void)pair_bytes; (void)l2;
-    int G = pin && *pin ? atoi(pin) : 1;
-    if (G < 1) G = 1;
-    if (G > 16) G = 16;
-    *resident_ctas = resident - resident % G;
-    *group_size = G;
-    return cudaSuccess;
+    if (dtype == METASD_BF16) return launch_streaming_t<__nv_bfloat16>(p, geo, stream, launches);
+    return launch_streaming_t<float>(p, geo, stream, launches);
 }
 
 // -------------------------------------------------------------------------------------------
-// drafter table check
+// reset
 // -------------------------------------------------------------------------------------------
-// Copies the caller's table of K drafter pointers into the context's own table.  An entry that is NULL or not
-// aligned like the target (16 bytes on the vector path, else the element size) must never be dereferenced: it is
-// flagged and replaced by the target pointer, so that the outputs of the sequences that play that drafter are
-// defined (if meaningless) and nothing faults.
-__global__ void sanitize_table_kernel(const void *const *table, int K, const void *target, uint32_t mask,
-                                      const void **clean, uint32_t *status)
-{
-    const int i = threadIdx.x;
-    if (i >= K) return;
-    const void *q = table[i];
-    if (q == nullptr || (reinterpret_cast<uintptr_t>(q) & mask) != 0) {
-        atomicOr(status, METASD_STATUS_BAD_POINTER);
-        q = target;
-    }
-    clean[i] = q;
-}
-
-cudaError_t launch_sanitize_table(const void *const *table, int K, const void *target, uint32_t mask, const void **clean,
-                                  uint32_t *status, cudaStream_t stream)
-{
-    sanitize_table_kernel<<<1, 32, 0, stream>>>(table, K, target, mask, clean, status);
-    return cudaGetLastError();
-}
-
-// -------------------------------------------------------------------------------------------
-// select / reset
-// -------------------------------------------------------------------------------------------
-__global__ void select_kernel(BanditState st, int batch, int32_t *arm_out)
-{
-    int b = blockIdx.x * blockDim.x + threadIdx.x;
-    if (b < batch) arm_out[b] = st.arm[b];
-}
-
 __global__ void reset_kernel(BanditState st, int max_batch, int K, int tau, int variant, double gamma,
                              uint32_t sequence_base, const int32_t *seq_ids, int n)
 {
@@ -1130,12 +979,6 @@ __global__ void reset_kernel(BanditState st, int max_batch, int K, int tau, int 
                                   st.win_arm + (size_t)b * tau, st.win_reward + (size_t)b * tau, 0ull,
                                   sequence_base + (uint32_t)b);
     }
-}
-
-cudaError_t launch_select(const BanditState &st, int batch, int32_t *arm_out, cudaStream_t stream)
-{
-    select_kernel<<<(batch + 255) / 256, 256, 0, stream>>>(st, batch, arm_out);
-    return cudaGetLastError();
 }
 
 cudaError_t launch_reset(const BanditState &st, int max_batch, int K, int tau, int variant, double gamma,

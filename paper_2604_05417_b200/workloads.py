@@ -7,8 +7,11 @@ both receive the exact bytes produced here.
 Recipe (stand-in for the paper's Vicuna-7B target + task-specialised drafters,
 whose weights and datasets are not available):
 
-* target[b, j, v] = round(dtype, 3 * z - s_b * ln(v + 1)),  z ~ N(0, 1) i.i.d.
-  (a Zipf(s_b) log-prior over token ids plus Gaussian noise of std 3)
+* target[b, j, v] = round(dtype, 3 * z - s_b * ln(rank(v))),  z ~ N(0, 1) i.i.d.
+  (a Zipf(s_b) log-prior over token ids plus Gaussian noise of std 3).  rank(v) = v + 1 by default (the likely
+  tokens have the small ids, as in a frequency-sorted vocabulary); ``order="reversed"`` puts them at the END of the
+  vocabulary and ``order="shuffled"`` spreads them by a seeded permutation, so that an implementation that walks the
+  vocabulary in id order cannot profit from where the mass sits.
 * draft[b, j, v]  = round(dtype, float(target[b, j, v]) + sigma * z'),  z' ~ N(0, 1)
   where sigma is the noise level of the drafter that produced the block; a
   better-aligned drafter has a smaller sigma.
@@ -49,6 +52,7 @@ class Workload:
     beta: float = 0.01
     gamma: float = 0.975
     tau: int = 50
+    order: str = "rank"         # which token ids are the likely ones: "rank" | "reversed" | "shuffled"
 
     def scaled(self, **kw) -> "Workload":
         return replace(self, **kw)
@@ -108,6 +112,13 @@ class RoundGenerator:
             chunk_sequences = max(1, min(wl.B, (1 << 30) // per_seq))
         self.chunk = chunk_sequences
         v = torch.arange(1, wl.V + 1, dtype=torch.float32, device=self.device)
+        if wl.order == "reversed":
+            v = v.flip(0)
+        elif wl.order == "shuffled":
+            perm = np.random.RandomState(_seed(seed, 77) % (2 ** 32)).permutation(wl.V)
+            v = v[torch.from_numpy(perm).to(self.device)]
+        elif wl.order != "rank":
+            raise ValueError(wl.order)
         self._log_rank = torch.log(v)
         zipf = np.asarray([wl.zipf[b % len(wl.zipf)] for b in range(wl.B)], dtype=np.float32)
         self._zipf = torch.from_numpy(zipf).to(self.device)

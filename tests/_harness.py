@@ -11,6 +11,9 @@ Comparison rules (what "results identical to the oracle" means here):
 """
 from __future__ import annotations
 
+import json
+import os
+
 import numpy as np
 import torch
 
@@ -34,12 +37,12 @@ def new_context(*args, **kw):
 
 
 def make_pair(wl: Workload, path=M.PATH_AUTO, reward=M.REWARD_BD, bandit=None, device=0, sequence_base=0,
-              beta=None, host_staging=False):
+              beta=None, host_staging=False, **tuning):
     bandit = bandit or wl.bandit
     beta = wl.beta if beta is None else beta
     gpu = new_context(wl.B, wl.N, wl.k, wl.V, dtype=wl.dtype, bandit=bandit, beta=beta, gamma=wl.gamma,
                       window=wl.tau, reward=reward, device=device, path=path, sequence_base=sequence_base,
-                      host_staging=host_staging)
+                      host_staging=host_staging, **tuning)
     orc = O.OracleMetaSD(O.OracleConfig(max_batch=wl.B, n_drafters=wl.N, vocab=wl.V, bandit=M.BANDITS[bandit],
                                         beta=beta, gamma=wl.gamma, tau=wl.tau, reward=reward,
                                         sequence_base=sequence_base))
@@ -103,12 +106,11 @@ def compare_round(res, out, target, draft, T, reward_T, counts):
     tok_mism = ok & (g_tok != out["next_token"])
     if tok_mism.any():
         assert not greedy, "greedy tokens must be bit-exact"
-        tgt = target.float().cpu().numpy().astype(np.float64)
-        drf = draft.float().cpu().numpy().astype(np.float64)
         for b in np.nonzero(tok_mism)[0]:
             assert out["sample_margin"][b] < NEAR, "sampled token differs away from a CDF edge"
             j = int(out["accepted_len"][b])
-            w = _row_weights(tgt[b, j], drf[b, j] if j < k else None, T)
+            row = lambda x: x.float().cpu().numpy().astype(np.float64)
+            w = _row_weights(row(target[b, j]), row(draft[b, j]) if j < k else None, T)
             # the two tokens must be neighbours in the CDF: what lies strictly between them carries (next to) no mass.
             # In float64 that is "the neighbouring token with mass"; fp32 may flush weights of 1e-12 that float64
             # still sees, so the bound is on the mass in between, not on the count of tokens.
@@ -126,15 +128,42 @@ def reward_kind_is_bd(out, k):
     return out.get("_reward_kind", M.REWARD_BD) == M.REWARD_BD
 
 
+def gather_by_arm(drafts, tokens, arm, dev):
+    """Rows and tokens of the drafter each sequence plays, picked out of the K per-drafter tensors (input
+    marshalling for the oracle, which then reads [B,k,V] instead of K such tensors)."""
+    idx = torch.as_tensor(arm, device=dev, dtype=torch.long)
+    draft = torch.empty_like(drafts[0])
+    toks = torch.empty_like(tokens[0])
+    for i in range(len(drafts)):
+        rows = torch.nonzero(idx == i).flatten()
+        if rows.numel():
+            draft[rows] = drafts[i][rows]
+            toks[rows] = tokens[i][rows]
+    return draft, toks
+
+
+def write_report(label: str, counts: dict):
+    """Appends the counters of a lock-step run to the JSON-lines file named by METASD_PARITY_REPORT (if set)."""
+    path = os.environ.get("METASD_PARITY_REPORT")
+    if not path:
+        return
+    row = {"case": label}
+    row.update({k: (v if isinstance(v, (int, float, str)) else float(v)) for k, v in counts.items()})
+    with open(path, "a") as f:
+        f.write(json.dumps(row) + "\n")
+
+
 def run_lockstep(wl: Workload, rounds: int, seed: int = 0, lib_seed: int = 1234, path=M.PATH_AUTO,
                  reward=M.REWARD_BD, bandit=None, table_mode=False, device=0, sequence_base=0, beta=None,
-                 check_state=True):
-    """Runs `rounds` rounds of the workload on both sides and compares every round."""
+                 check_state=True, oracle_reads_tables=True, label=None, **tuning):
+    """Runs `rounds` rounds of the workload on both sides and compares every round.  table_mode: the library reads
+    the K drafters' tensors through its pointer table; the oracle then reads the same tables, or (for the large
+    configurations, oracle_reads_tables=False) the rows gathered by its own arm choice."""
     dev = torch.device("cuda", device)
     gen = RoundGenerator(wl, device=dev, seed=seed)
     gpu, orc = make_pair(wl, path=path, reward=reward, bandit=bandit, device=device,
-                         sequence_base=sequence_base, beta=beta)
-    counts = {}
+                         sequence_base=sequence_base, beta=beta, **tuning)
+    counts = {"sequences": wl.B, "near_tie_accept": 0, "near_tie_token": 0, "near_tie_arm": 0, "best_arm_plays": 0}
     T = wl.temperature
     try:
         for t in range(rounds):
@@ -152,17 +181,19 @@ def run_lockstep(wl: Workload, rounds: int, seed: int = 0, lib_seed: int = 1234,
                 table = M.pointer_table(rd["drafts"])
                 res = gpu.verify(rd["target"], None, rd["tokens"], T, lib_seed, drafter_table=table,
                                  token_arm_stride=wl.B * wl.k, want_diag=True)
-                idx = torch.as_tensor(arm_o, device=dev, dtype=torch.long)
-                draft = torch.stack(rd["drafts"])[idx, torch.arange(wl.B, device=dev)]
-                tokens = rd["tokens"][idx, torch.arange(wl.B, device=dev)]
-                out = orc.verify(rd["target"], None, tokens.cpu().numpy(), T, lib_seed,
-                                 drafter_tables=rd["drafts"])
+                draft, tokens = gather_by_arm(rd["drafts"], rd["tokens"], arm_o, dev)
+                if oracle_reads_tables:
+                    out = orc.verify(rd["target"], None, tokens.cpu().numpy(), T, lib_seed,
+                                     drafter_tables=rd["drafts"])
+                else:
+                    out = orc.verify(rd["target"], draft, tokens.cpu().numpy(), T, lib_seed)
             else:
                 rd = gen.gathered_round(t, arm_o)
                 draft = rd["draft"]
                 res = gpu.verify(rd["target"], draft, rd["tokens"], T, lib_seed, want_diag=True)
                 out = orc.verify(rd["target"], draft, rd["tokens"].cpu().numpy(), T, lib_seed)
             out["_reward_kind"] = reward
+            counts["best_arm_plays"] += int((arm_o == gen.best_arm(t)).sum())
             diverged = compare_round(res, out, rd["target"], draft, T, 1.0, counts)
             if diverged.any() and reward == M.REWARD_BE:
                 gpu.state_import(oracle_state_blob(orc))   # BE feeds accept bits into the bandit
@@ -177,6 +208,8 @@ def run_lockstep(wl: Workload, rounds: int, seed: int = 0, lib_seed: int = 1234,
         counts["status"] = gpu.last_status()
         counts["launches"] = gpu.kernel_launches()
         counts["path"] = gpu.resolved_path(wl.k)
+        counts["row_kernel"] = gpu.resolved_row_kernel()
     finally:
         gpu.close()
+    write_report(label or wl.name, counts)
     return counts

@@ -450,3 +450,160 @@ def test_full_size_launch_sampled_against_oracle(name, path):
                 if T == 0 or out["sample_margin"][0] > 1e-6:
                     assert res.next_token[b].item() == out["next_token"][0]
     gpu.close()
+
+
+# ------------------------------------------------------------------------------------------------------------------
+# The five benchmark configurations at their full batch, every sequence in lock-step with the oracle, well past the
+# initial sweep, the bandit choosing the drafter through the pointer table.
+# ------------------------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("bandit", ["ducb", "swucb"])
+def test_cfg2_full_batch_nonstationary(bandit):
+    """All 64 sequences, 250 rounds at the real period of 100: the drafter noise is re-permuted twice, and the
+    discounted / sliding-window statistics follow the oracle's through both changes."""
+    from _harness import run_lockstep
+    wl = WORKLOADS["cfg2_nonstationary"]
+    c = report(run_lockstep(wl, rounds=250, bandit=bandit, table_mode=True, label="cfg2_full_%s" % bandit))
+    assert c["rounds"] == 250 and c["sequences"] == 64 and c["near_tie_arm"] == 0 and c["status"] == 0
+    assert c["best_arm_plays"] > 0.3 * 250 * 64     # the policies do track the moving best drafter
+
+
+def test_cfg3_full_batch():
+    from _harness import run_lockstep
+    wl = WORKLOADS["cfg3_tasks"]
+    c = report(run_lockstep(wl, rounds=30, table_mode=True, oracle_reads_tables=False, label="cfg3_full"))
+    assert c["rounds"] == 30 and c["sequences"] == 256 and c["near_tie_arm"] == 0 and c["status"] == 0
+
+
+def test_cfg4_full_batch_greedy_bit_exact():
+    from _harness import run_lockstep
+    wl = WORKLOADS["cfg4_greedy"]
+    c = report(run_lockstep(wl, rounds=24, table_mode=True, oracle_reads_tables=False, label="cfg4_full"))
+    assert c["rounds"] == 24 and c["sequences"] == 512 and c["status"] == 0
+    assert c["near_tie_accept"] == 0 and c["near_tie_token"] == 0 and c["near_tie_arm"] == 0
+
+
+@pytest.mark.parametrize("bandit", ["ucb", "ducb"])
+def test_cfg5_full_batch(bandit):
+    from _harness import run_lockstep
+    wl = WORKLOADS["cfg5_fp32_stress"]
+    c = report(run_lockstep(wl, rounds=20, bandit=bandit, table_mode=True, oracle_reads_tables=False,
+                            label="cfg5_full_%s" % bandit))
+    assert c["rounds"] == 20 and c["sequences"] == 1024 and c["near_tie_arm"] == 0 and c["status"] == 0
+
+
+# ------------------------------------------------------------------------------------------------------------------
+# Every row-statistics variant and the draw's early stop
+# ------------------------------------------------------------------------------------------------------------------
+ROW_KERNELS = [dict(row_kernel=M.ROWS_PLAIN), dict(row_kernel=M.ROWS_STAGED),
+               dict(row_kernel=M.ROWS_STAGED, row_threads=1024, row_stages=6),
+               dict(row_kernel=M.ROWS_BULK), dict(row_kernel=M.ROWS_BULK, row_threads=512, row_stages=3),
+               dict(row_kernel=M.ROWS_BULK, row_threads=1024, row_stages=7),
+               dict(row_kernel=M.ROWS_BULK, row_threads=768, row_stages=8)]
+
+
+@pytest.mark.parametrize("tuning", ROW_KERNELS, ids=lambda d: "-".join(str(v) for v in d.values()))
+@pytest.mark.parametrize("dtype,V,T", [("bf16", 152064, 0.0), ("bf16", 50264, 1.3), ("fp32", 128256, 1.0),
+                                       ("bf16", 8200, 0.8), ("fp32", 1000, 1.0), ("bf16", 32000, 1.0)])
+def test_row_kernel_variants(tuning, dtype, V, T):
+    """Plain loads, per-thread staged copies and the bulk-copy ring give the oracle's round at vocabularies from
+    less than one chunk to many trips of every ring depth, with a ragged last chunk."""
+    from _harness import run_lockstep
+    wl = base(B=10, N=3, k=4, V=V, sigmas=(0.3, 1.0, 2.5)).scaled(dtype=dtype, temperature=T)
+    c = report(run_lockstep(wl, rounds=6, seed=V % 89, path=M.PATH_STREAMING, table_mode=True, **tuning))
+    assert c["rounds"] == 6 and c["status"] == 0 and c["row_kernel"] == tuning["row_kernel"]
+    if T == 0.0:
+        assert c["near_tie_accept"] == 0 and c["near_tie_token"] == 0 and c["near_tie_arm"] == 0
+
+
+@pytest.mark.parametrize("tuning", [dict(row_kernel=M.ROWS_STAGED), dict(row_kernel=M.ROWS_BULK)],
+                         ids=["staged", "bulk"])
+def test_row_kernels_with_per_sequence_draft_lengths_and_odd_logit_scales(tuning):
+    """The bulk-copy kernel skips positions behind a sequence's draft length and redoes a draft row whose sum the
+    shared reference flushed, like the staged kernel does."""
+    from _harness import make_pair, compare_round
+    wl = base(B=9, N=1, k=4, V=30000, sigmas=(0.8,)).scaled(temperature=0.9)
+    dev = torch.device("cuda", 0)
+    gen = RoundGenerator(wl, device=dev, seed=21)
+    gpu, orc = make_pair(wl, path=M.PATH_STREAMING, **tuning)
+    offsets = torch.tensor([0.0, -150.0, 150.0, -70.0, 70.0, -110.0, 110.0, 20.0, 0.0], device=dev)
+    lens = np.array([4, 1, 2, 3, 4, 2, 1, 3, 4], dtype=np.int32)
+    lens_dev = torch.from_numpy(lens).to(dev)
+    gpu.set_draft_lengths(lens_dev)
+    counts = {}
+    try:
+        for t in range(3):
+            arm = orc.select()
+            rd = gen.gathered_round(t, arm)
+            draft = (rd["draft"].float() + offsets.view(-1, 1, 1)).to(rd["draft"].dtype)
+            target = rd["target"].clone()
+            for b in range(wl.B):
+                target[b, lens[b] + 1:] = float("nan")
+                draft[b, lens[b]:] = float("nan")
+            res = gpu.verify(target, draft, rd["tokens"], 0.9, 31, want_diag=True)
+            out = orc.verify(target, draft, rd["tokens"].cpu().numpy(), 0.9, 31, draft_len=lens)
+            assert gpu.last_status() == 0 and (out["status"] == 0).all()
+            assert np.array_equal(res.accepted_len.cpu().numpy(), out["accepted_len"])
+            np.testing.assert_allclose(res.reward.cpu().numpy(), out["reward"], rtol=0, atol=1e-5)
+            D = res.diag_fields()[2].cpu().numpy()
+            for b in range(wl.B):
+                np.testing.assert_allclose(D[b, :lens[b]], out["D"][b, :lens[b]], rtol=0, atol=1e-5)
+            firm = out["sample_margin"] > 1e-6
+            assert np.array_equal(res.next_token.cpu().numpy()[firm], out["next_token"][firm])
+    finally:
+        gpu.close()
+
+
+@pytest.mark.parametrize("order", ["rank", "reversed", "shuffled"])
+@pytest.mark.parametrize("dtype,V", [("bf16", 152064), ("fp32", 50264), ("bf16", 600)])
+def test_draw_stops_at_the_crossing_wherever_the_mass_sits(order, dtype, V):
+    """The inverse-CDF draw walks the vocabulary in id order and stops behind the crossing.  With the likely tokens
+    at the END of the vocabulary (reversed) it has to walk the whole row, with shuffled ids about half of it: the
+    drawn tokens are the oracle's in every case."""
+    from _harness import run_lockstep
+    wl = base(B=24, N=3, k=3, V=V, sigmas=(0.2, 1.0, 3.0)).scaled(dtype=dtype, temperature=1.0, order=order)
+    c = report(run_lockstep(wl, rounds=8, seed=5, path=M.PATH_STREAMING, table_mode=True))
+    assert c["rounds"] == 8 and c["status"] == 0
+
+
+def test_a_device_wait_that_runs_out_sets_the_timeout_bit_and_the_call_still_ends():
+    """wait_poll_limit = 1 makes the consumers of the bulk-copy ring give up on the first chunk that has not landed
+    when they look: the call ends, the status word carries METASD_STATUS_TIMEOUT (its outputs are undefined), and
+    the device keeps working -- a context with the default limit gives the oracle's round right after."""
+    from _harness import run_lockstep
+    wl = base(B=6, N=2, k=3, V=152064, sigmas=(0.5, 2.0))
+    dev = torch.device("cuda", 0)
+    gen = RoundGenerator(wl, device=dev, seed=2)
+    gpu = M.MetaSD(wl.B, wl.N, wl.k, wl.V, row_kernel=M.ROWS_BULK, wait_poll_limit=1)
+    rd = gen.gathered_round(0, np.zeros(wl.B, dtype=np.int64))
+    res = gpu.verify(rd["target"], rd["draft"], rd["tokens"], 1.0, 4)
+    torch.cuda.synchronize()
+    assert gpu.last_status() & M.STATUS_TIMEOUT
+    assert res.accepted_len.shape == (wl.B,)
+    gpu.reset()
+    gpu.close()
+    c = run_lockstep(wl, rounds=3, path=M.PATH_STREAMING, row_kernel=M.ROWS_BULK)
+    assert c["status"] == 0 and c["rounds"] == 3
+
+
+def test_state_import_refuses_out_of_range_values_before_they_reach_the_device():
+    gpu = M.MetaSD(4, 3, 2, 1024, bandit="swucb", window=6)
+    parts = M.parse_state(gpu.state_export(), 4, 3, 6)
+    for field, index, value in [("arm", 2, 3), ("arm", 0, -1), ("t", 1, -5), ("win_arm", (3, 5), 99),
+                                ("stat_b", (0, 0), float("nan"))]:
+        bad = {k: np.array(v, copy=True) for k, v in parts.items()}
+        bad[field][index] = value
+        with pytest.raises(M.MetasdError) as e:
+            gpu.state_import(M.pack_state(bad))
+        assert e.value.code == M.ERR_BAD_STATE_BLOB
+    gpu.state_import(M.pack_state(parts))            # the untouched blob is accepted
+    assert gpu.state_export() == M.pack_state(parts)
+    gpu.close()
+
+
+def test_context_calls_run_on_the_contexts_device_and_leave_the_callers_current_device_alone():
+    dev = torch.device("cuda", 0)
+    before = torch.cuda.current_device()
+    gpu = M.MetaSD(2, 2, 2, 512, device=0)
+    gpu.select()
+    assert torch.cuda.current_device() == before
+    gpu.close()

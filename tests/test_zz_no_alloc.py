@@ -4,9 +4,10 @@
 owns the device, a plugin that may not allocate after start-up -- and therefore cannot create a
 context.  Its scratch is a fixed array inside the library.  This test drives it through the C ABI on
 two consecutive rounds and checks that it returns what `metasd_verify` returns for the same inputs,
-seed, sequence ids and round counters: integers exactly, the reward within the 1e-5 the parity tests
-use.  It builds its own contexts and inputs, so it passes alone in a fresh process as well as after
-the rest of the suite.
+seed, sequence ids and round counters, and what the float64 CPU oracle computes for them: integers
+exactly (a sampled decision may differ only where the oracle itself marks it a near tie, as in the
+parity tests), the reward within the 1e-5 the parity tests use.  It builds its own contexts and inputs,
+so it passes alone in a fresh process as well as after the rest of the suite.
 """
 import numpy as np
 import pytest
@@ -25,7 +26,9 @@ def test_noalloc_matches_context_call_on_two_rounds(dtype, temperature, V):
     dev = torch.device("cuda", 0)
     torch.cuda.set_device(dev)
     gen = RoundGenerator(wl, device=dev, seed=17)
+    from oracle import oracle as O
     ctx = M.MetaSD(wl.B, 1, wl.k, V, dtype=dtype, path=M.PATH_STREAMING, sequence_base=40)
+    orc = O.OracleMetaSD(O.OracleConfig(max_batch=wl.B, n_drafters=1, vocab=V, sequence_base=40))
     acc = torch.full((wl.B,), -9, dtype=torch.int32, device=dev)
     tok = torch.full((wl.B,), -9, dtype=torch.int32, device=dev)
     rew = torch.full((wl.B,), -9.0, dtype=torch.float32, device=dev)
@@ -37,9 +40,23 @@ def test_noalloc_matches_context_call_on_two_rounds(dtype, temperature, V):
                               status=status, sequence_base=40)
         assert rc == M.OK
         torch.cuda.synchronize()
-        assert torch.equal(acc, want.accepted_len)
-        assert torch.equal(tok, want.next_token)
+        out = orc.verify(rd["target"], rd["draft"], rd["tokens"].cpu().numpy(), temperature, 31337)
+        assert (out["round"] == t).all()
+        with np.errstate(divide="ignore", invalid="ignore"):
+            firm = ~(np.abs(out["u_accept"] - out["p_x"] / out["q_x"]) < 1e-6).any(axis=1)
+        if temperature == 0:
+            firm[:] = True
+        firm_t = torch.from_numpy(firm).to(dev)
+        assert torch.equal(acc[firm_t], want.accepted_len[firm_t])
+        assert np.array_equal(acc.cpu().numpy()[firm], out["accepted_len"][firm])
+        if temperature > 0:
+            firm &= out["sample_margin"] > 1e-6
+            firm_t = torch.from_numpy(firm).to(dev)
+        assert torch.equal(tok[firm_t], want.next_token[firm_t])
+        assert np.array_equal(tok.cpu().numpy()[firm], out["next_token"][firm])
+        assert firm.sum() >= wl.B - 1
         assert torch.allclose(rew, want.reward, rtol=0, atol=1e-5)
+        np.testing.assert_allclose(rew.cpu().numpy(), out["reward"], rtol=0, atol=1e-5)
         assert status.item() == ctx.last_status()
     ctx.close()
 
