@@ -127,7 +127,7 @@ typedef struct metasd_config {
     int32_t fused_cluster;      /* METASD_PATH_FUSED: CTAs per cluster (0 = the smallest that fits) */
     int32_t fused_threads;      /* METASD_PATH_FUSED: threads per CTA (0 = chosen from the slice length) */
     int32_t wait_poll_limit;    /* polls after which a device-side wait on an asynchronous copy gives up and sets
-                                   METASD_STATUS_TIMEOUT (0 = about a quarter of a second).  For tests of that path. */
+                                   METASD_STATUS_TIMEOUT (0 = 2^18 polls of up to 4 us each: about a second).  For tests of that path. */
     int32_t reserved;           /* must be 0 */
 } metasd_config;
 

@@ -255,8 +255,8 @@ int metasd_select(metasd_ctx *ctx, int32_t batch, int32_t *arm_out, void *stream
 {
     if (!ctx || !arm_out || batch < 1 || batch > ctx->cfg.max_batch) return METASD_ERR_INVALID_ARGUMENT;
     ON_DEVICE_OF(ctx);
-    // the arm of the coming round was chosen at the end of the previous epilogue: the call is a copy
-    CK(cudaMemcpyAsync(arm_out, ctx->st.arm, (size_t)batch * sizeof(int32_t), cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
+    CK(launch_select(ctx->st, batch, arm_out, (cudaStream_t)stream));
+    ctx->launches += 1;
     return METASD_OK;
 }
 
@@ -305,7 +305,7 @@ int metasd_verify(metasd_ctx *ctx, int32_t batch, int32_t k, const void *target_
         const long long nvec = (long long)cfg.vocab * (long long)logit_size(cfg.logit_dtype) / 16;
         p.keep_from_vec = (int32_t)(nvec - nvec * ctx->keep_permille / 1000);
     }
-    p.poll_limit = cfg.wait_poll_limit > 0 ? (uint32_t)cfg.wait_poll_limit : (1u << 22);
+    p.poll_limit = cfg.wait_poll_limit > 0 ? (uint32_t)cfg.wait_poll_limit : (1u << 18);
     const size_t row_bytes = (size_t)cfg.vocab * logit_size(cfg.logit_dtype);
     // with a pointer table the per-drafter bases are not visible here: the kernels check every entry they use
     // against table_mask and never dereference one that fails

@@ -48,17 +48,32 @@ __device__ __forceinline__ bool mbar_test_wait(uint64_t *bar, uint32_t parity)
     return ok != 0;
 }
 
+// The suspending form of the wait with a time hint: the hardware parks the warp until the phase is over or about
+// `ns` nanoseconds have passed, so a warp that is ahead of its data costs one instruction, not a polling loop.
+__device__ __forceinline__ bool mbar_try_wait_for(uint64_t *bar, uint32_t parity, uint32_t ns)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_addr(bar)), "r"(parity), "r"(ns)
+        : "memory");
+    return ok != 0;
+}
+
 // Waits until the barrier's phase of the given parity is over, for at most `limit` polls.  Limits below 16 poll
-// without suspending the warp (so that a test can make a wait run out for certain); larger ones use the suspending
-// form and back off.  After a time-out every later wait of the CTA returns at once.
+// without suspending the warp (so that a test can make a wait run out for certain); larger ones park the warp for up
+// to 4 us per poll (the default limit of 2^18 polls, about a second, is far beyond any real wait and still ends).  After a time-out
+// every later wait of the CTA returns at once.
 __device__ __forceinline__ void wait_phase(uint64_t *bar, uint32_t parity, uint32_t limit, BulkShared &sh, uint32_t *status)
 {
-    const bool tiny = limit < 16u;
-    if (tiny ? mbar_test_wait(bar, parity) : mbar_try_wait(bar, parity)) return;
+    if (mbar_test_wait(bar, parity)) return;
     if (*(volatile int *)&sh.dead) return;
+    const bool tiny = limit < 16u;
     for (uint32_t it = 0; it < limit; ++it) {
-        if (tiny ? mbar_test_wait(bar, parity) : mbar_try_wait(bar, parity)) return;
-        if (it >= 128u) __nanosleep(64);
+        if (tiny ? mbar_test_wait(bar, parity) : mbar_try_wait_for(bar, parity, 4000u)) return;
     }
     *(volatile int *)&sh.dead = 1;
     atomicOr(status, METASD_STATUS_TIMEOUT);
@@ -175,7 +190,7 @@ __global__ void __launch_bounds__((NCW + 1) * 32, MINB) row_stats_bulk_kernel(co
         for (uint32_t g = fill - outstanding; g < fill; ++g) {
             uint64_t *bar = &sh.full[g % S];
             const uint32_t par = (g / S) & 1u;
-            for (uint32_t it = 0; it < (1u << 22) && !mbar_try_wait(bar, par); ++it) __nanosleep(64);
+            for (uint32_t it = 0; it < (1u << 20) && !mbar_try_wait(bar, par); ++it) __nanosleep(64);
         }
         return;
     }
@@ -361,14 +376,6 @@ static cudaError_t prepare_shape()
 {
     return cudaFuncSetAttribute(row_stats_bulk_kernel<LT, THREADS / 32 - 1, S, M>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 S * 2 * (THREADS - 32) * 16);
-}
-
-bool bulk_shape_built(int threads, int stages)
-{
-#define X(T, S, M) if (threads == T && stages == S) return true;
-    METASD_BULK_SHAPES(X)
-#undef X
-    return false;
 }
 
 cudaError_t bulk_prepare(int dtype, RowGeometry *geo)

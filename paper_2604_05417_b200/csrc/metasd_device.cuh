@@ -464,4 +464,90 @@ __device__ inline void bandit_update(int variant, int K, double gamma, int tau, 
     *t = *t + 1;
 }
 
+// bandit_update followed by bandit_select for one sequence, by one whole warp: for the UCB family (Algorithm 2, its
+// discounted and its sliding-window form) lane i holds arm i, so the fp64 divisions, square roots and the window
+// scan of the K arms run side by side; the arithmetic per arm, the order of the window's additions and the
+// lowest-index tie-break are those of the serial functions.  The other policies run on lane 0.  Returns the next arm
+// (the same value in every lane) after storing it and the advanced round counter.
+__device__ inline int warp_bandit_step(int variant, int K, double beta, double gamma, int tau, int32_t *t_ptr, int32_t *arm_ptr,
+                                       double *sa, double *sb, int32_t *wa, double *wr, int a, double r, uint64_t seed,
+                                       uint32_t sequence)
+{
+    const int lane = threadIdx.x & 31;
+    const int t = *t_ptr;
+    int next = 0;
+    if (variant != METASD_UCB && variant != METASD_DUCB && variant != METASD_SWUCB) {
+        if (lane == 0) {
+            int32_t tt = t;
+            bandit_update(variant, K, gamma, tau, &tt, sa, sb, wa, wr, a, r);
+            next = bandit_select(variant, K, beta, gamma, tau, tt, sa, sb, wa, wr, seed, sequence);
+            *t_ptr = tt;
+            *arm_ptr = next;
+        }
+        return __shfl_sync(0xFFFFFFFFu, next, 0);
+    }
+    double a_i = 0.0, b_i = 0.0;
+    if (variant == METASD_UCB) {
+        if (lane < K) { a_i = sa[lane]; b_i = sb[lane]; }
+        if (lane == a) {
+            a_i = (a_i * b_i + r) / (b_i + 1.0);
+            b_i = b_i + 1.0;
+            sa[lane] = a_i;
+            sb[lane] = b_i;
+        }
+    } else if (variant == METASD_DUCB) {
+        if (lane < K) {
+            a_i = sa[lane] * gamma;
+            b_i = sb[lane] * gamma;
+            if (lane == a) { a_i += r; b_i += 1.0; }
+            sa[lane] = a_i;
+            sb[lane] = b_i;
+        }
+    } else {
+        if (lane == 0) {
+            const int slot = t % tau;
+            wa[slot] = a;
+            wr[slot] = r;
+        }
+        __syncwarp();
+    }
+    const int t1 = t + 1;
+    next = t1;   // initial sweep: every drafter once, in order
+    if (t1 >= K) {
+        double mu = 0.0, n = 0.0;
+        if (variant == METASD_SWUCB) {
+            if (lane < K) {
+                const int first = t1 - tau > 0 ? t1 - tau : 0;
+                for (int s = first; s < t1; ++s) {   // oldest first
+                    const int slot = s % tau;
+                    if (wa[slot] == lane) { mu += wr[slot]; n += 1.0; }
+                }
+                if (n > 0.0) mu /= n;
+            }
+        } else if (variant == METASD_DUCB) {
+            n = b_i;
+            mu = a_i / b_i;
+        } else {
+            mu = a_i;
+            n = b_i;
+        }
+        const double two_ln_t = 2.0 * log((double)t1);
+        double score = -INFINITY;
+        if (lane < K) score = n > 0.0 ? mu + beta * sqrt(two_ln_t / n) : INFINITY;
+        int best = lane;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const double os = __shfl_xor_sync(0xFFFFFFFFu, score, o);
+            const int ob = __shfl_xor_sync(0xFFFFFFFFu, best, o);
+            if (os > score || (os == score && ob < best)) { score = os; best = ob; }
+        }
+        next = best;
+    }
+    if (lane == 0) {
+        *t_ptr = t1;
+        *arm_ptr = next;
+    }
+    return next;
+}
+
 }  // namespace metasd

@@ -73,7 +73,6 @@ struct VerifyParams {
 // streaming path (metasd_streaming.cu, metasd_bulk.cu)
 cudaError_t streaming_prepare(int device, int dtype, const metasd_config &cfg, RowGeometry *geo);
 cudaError_t launch_streaming(const VerifyParams &p, int dtype, const RowGeometry &geo, cudaStream_t stream, uint64_t *launches);
-bool bulk_shape_built(int threads, int stages);
 cudaError_t bulk_prepare(int dtype, RowGeometry *geo);
 cudaError_t launch_row_stats_bulk(const VerifyParams &p, int dtype, const RowGeometry &geo, cudaStream_t stream);
 // fused cluster path (metasd_fused.cu)
@@ -93,6 +92,7 @@ cudaError_t fused_prepare(int device, int dtype, int V, int max_batch, int pin_c
 cudaError_t launch_fused(const VerifyParams &p, int dtype, const FusedPlan &plan, cudaStream_t stream,
                          uint64_t *launches);
 // small state kernels (metasd_streaming.cu)
+cudaError_t launch_select(const BanditState &st, int batch, int32_t *arm_out, cudaStream_t stream);
 cudaError_t launch_reset(const BanditState &st, int max_batch, int K, int tau, int variant, double gamma,
                          uint32_t sequence_base, const int32_t *seq_ids, int n, cudaStream_t stream);
 

@@ -140,7 +140,7 @@ extern "C" int metasd_verify_noalloc(int32_t batch, int32_t k, int32_t vocab, in
         const long long nvec = (long long)row_bytes / 16;
         p.keep_from_vec = (int32_t)(nvec - nvec * (logit_dtype == METASD_BF16 ? 750 : 900) / 1000);
     }
-    p.poll_limit = 1u << 22;
+    p.poll_limit = 1u << 18;
 
     noalloc_prepare_kernel<<<(batch + 255) / 256, 256, 0, s>>>(batch, (int32_t)round);
     cudaError_t e = cudaGetLastError();

@@ -457,12 +457,11 @@ __device__ __forceinline__ void draw_weights(const LT *a, const LT *d, int i, in
 }
 
 // Sum of the draw's weights over the vectors [lo, hi), by one warp: lane l takes lo + l, lo + l + 32, ... and adds
-// each vector's fp32 sum to its fp64 total in that order.  Four vectors' loads are issued before the first is used.
-template <typename LT, int VEC, int MODE>
+// each vector's fp32 sum to its fp64 total in that order.  U vectors' loads are issued before the first is used.
+template <typename LT, int VEC, int MODE, int U>
 __device__ __forceinline__ double warp_range_sum_m(const LT *a, const LT *d, int lo, int hi, float c, float nma,
                                                    float ia, float nmb, float ib)
 {
-    constexpr int U = 4;
     const int lane = threadIdx.x & 31;
     double acc = 0.0;
     for (int i0 = lo + lane; i0 < hi; i0 += 32 * U) {
@@ -493,12 +492,12 @@ __device__ __forceinline__ double warp_range_sum_m(const LT *a, const LT *d, int
     return warp_sum(acc);
 }
 
-template <typename LT, int VEC>
+template <typename LT, int VEC, int U = 4>
 __device__ __forceinline__ double warp_range_sum(const LT *a, const LT *d, int lo, int hi, int mode, float c,
                                                  float nma, float ia, float nmb, float ib)
 {
-    return mode == 1 ? warp_range_sum_m<LT, VEC, 1>(a, d, lo, hi, c, nma, ia, nmb, ib)
-                     : warp_range_sum_m<LT, VEC, 2>(a, d, lo, hi, c, nma, ia, nmb, ib);
+    return mode == 1 ? warp_range_sum_m<LT, VEC, 1, U>(a, d, lo, hi, c, nma, ia, nmb, ib)
+                     : warp_range_sum_m<LT, VEC, 2, U>(a, d, lo, hi, c, nma, ia, nmb, ib);
 }
 
 // Given n <= 64 non-negative parts x[0..n) laid end to end after base0, finds the first part whose end lies beyond
@@ -542,38 +541,49 @@ __device__ __forceinline__ int warp_find_part(const double *x, int n, double bas
 }
 
 // Shared-memory work space of the draw.
-constexpr int DRAW_MAX_SEG = 64;
 template <int NWARP> struct DrawShared {
-    double tot[2][NWARP];            // warp totals of a segment, double-buffered by segment parity
-    double sub[NWARP];               // warp totals of the second search level
-    double seg[DRAW_MAX_SEG];        // weight of every segment walked so far
+    double tot[NWARP], sub[NWARP];   // warp totals of the two search levels
     double before;                   // weight in front of the token that was found
     int tok;
 };
 
-// Second search level: the smallest token v in the vectors [r0, r1) with base + sum_{w in range, w <= v} weight_w >
-// threshold; rounding may leave none, then the last token of the range with mass (-1 if it has none).  Every warp
-// sums a part of the range, one warp-parallel scan finds the part that holds the crossing and the owning warp
-// finishes with a lane scan.  `before` receives base + the weight in front of the token.  The whole CTA takes part.
-template <typename LT, int VEC, int NWARP>
-__device__ int locate_in_range(const LT *a, const LT *d, int r0, int r1, int mode, float c, float nma, float ia, float nmb,
-                               float ib, double base, double threshold, DrawShared<NWARP> &sh, double &before)
+// Inverse CDF in token order over the vectors [0, v_end) of one row (pair): the smallest token v with
+// sum_{w <= v} weight_w > threshold.  Every warp owns a contiguous range of vectors and sums it (fp32 weights, fp64
+// sums); one warp-parallel scan finds the range that holds the crossing, the same two steps repeat inside that range,
+// and the owning warp finishes with a lane scan.  FRACTION: the threshold comes in as a fraction of the range's total
+// (the walk's own total, when the range is the whole row) and rounding may leave no crossing: then the last token
+// with mass.  Otherwise it is absolute, and -2 says that the crossing lies behind the range.  Returns the token (-1:
+// the range has no mass), the weight in front of it in `before` and the weight of the range in `total`.
+template <typename LT, int VEC, int NWARP, bool FRACTION>
+__device__ __forceinline__ int range_inverse_cdf(const LT *a, const LT *d, int v_end, int mode, double threshold, float c,
+                                                 float nma, float ia, float nmb, float ib, DrawShared<NWARP> &sh,
+                                                 double &before, double &total)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int per_warp = (v_end + NWARP - 1) / NWARP;
+    const int v0 = min(warp * per_warp, v_end), v1 = min(v0 + per_warp, v_end);
+    const double acc = warp_range_sum<LT, VEC>(a, d, v0, v1, mode, c, nma, ia, nmb, ib);
+    if (lane == 0) sh.tot[warp] = acc;
+    if (tid == 0) { sh.tok = -1; sh.before = 0.0; }
+    __syncthreads();
+    double base;
+    const int wstar = warp_find_part<FRACTION>(sh.tot, NWARP, 0.0, threshold, base, total);
+    if (!(total > 0.0) || wstar < 0) { before = 0.0; return -1; }
+    if (!FRACTION && !(total > threshold)) { before = total; return -2; }   // the crossing is not inside the range
+    const int r0 = min(wstar * per_warp, v_end), r1 = min(r0 + per_warp, v_end);
     const int per_sub = (r1 - r0 + NWARP - 1) / NWARP;
     const int s0 = min(r0 + warp * per_sub, r1), s1 = min(s0 + per_sub, r1);
     {
         const double acc2 = warp_range_sum<LT, VEC>(a, d, s0, s1, mode, c, nma, ia, nmb, ib);
         if (lane == 0) sh.sub[warp] = acc2;
-        if (tid == 0) { sh.tok = -1; sh.before = base; }
     }
     __syncthreads();
-    double total2, sub_base;
-    const int sstar = warp_find_part<false>(sh.sub, NWARP, base, threshold, sub_base, total2);
+    double total2;
+    const int sstar = warp_find_part<false>(sh.sub, NWARP, base, threshold, base, total2);
     if (warp == sstar) {
         int found = -1, last_pos = -1;
-        double found_before = sub_base, last_before = sub_base;
-        double run_base = sub_base;
+        double found_before = base, last_before = base;
+        double run_base = base;
         for (int i0 = s0; i0 < s1 && found < 0; i0 += 32) {
             const int i = i0 + lane;
             float w[VEC];
@@ -609,7 +619,6 @@ __device__ int locate_in_range(const LT *a, const LT *d, int r0, int r1, int mod
                         if (tok < 0 && cum + (double)w[e] > threshold) { tok = i * VEC + e; found_before = cum; }
                         cum += (double)w[e];
                     }
-                    // the vector's own sum crossed, so an element does unless rounding interferes
                     if (tok < 0) { tok = last_pos; found_before = last_before; }
                     found = tok;
                 }
@@ -618,7 +627,7 @@ __device__ int locate_in_range(const LT *a, const LT *d, int r0, int r1, int mod
             }
             run_base += __shfl_sync(0xFFFFFFFFu, incl, 31);
         }
-        if (found < 0) {  // rounding left the running sum a hair under the threshold: the last token with mass
+        if (found < 0) {
             int best = last_pos;
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) best = max(best, __shfl_xor_sync(0xFFFFFFFFu, best, o));
@@ -633,89 +642,56 @@ __device__ int locate_in_range(const LT *a, const LT *d, int r0, int r1, int mod
     return sh.tok;
 }
 
-// Inverse CDF in token order over one row (pair): the smallest v with sum_{w<=v} weight_w > u * total, where total is
-// the sum of all the weights as this walk adds them up (fp32 weights, fp64 sums).  The walk goes through the row in
-// token order, one segment at a time with the whole CTA on the segment, and stops behind the segment that holds the
-// crossing: `approx_total` is the total as the row statistics already give it (1 - sum_v min(p_v, q_v) for the
-// residual, 1 for the bonus row), equal to the walk's own total to within `guard`.  A token is taken early only if
-// it is the answer for every total in approx_total +- guard; otherwise (a CDF edge inside that band, or a total too
-// small for the band to mean anything) the walk goes on to the end of the row and decides with its own total.  The
-// answer is therefore always the one of the full walk.  Returns -1 when the row has no mass.
+// The draw of one sequence: the smallest v with sum_{w<=v} weight_w > u * total, total being the sum of all the weights
+// as the walk over the whole row adds them up.  `approx_total` is the same total as the row statistics already give
+// it (1 - sum_v min(p_v, q_v) for the residual, 1 for the bonus row); the two are fp32 evaluations of one sum and
+// agree to within `guard` (they were never seen further apart than 2e-6, typically 2e-7, over millions of rows).
+// So the first eighth of the vocabulary is searched first, with the upper end of the band u * (approx_total +- guard)
+// as the threshold: a token found there whose weight in front does not reach the lower end of the band is the answer
+// for every total in the band, hence the full walk's answer, and the rest of the row is never read.  Otherwise (the
+// crossing lies further back, a CDF edge falls inside the band, or the total is too small for the band to mean
+// anything) the whole row is walked and its own total decides.  With a frequency-sorted vocabulary most draws end in
+// the probe; with the likely tokens at the end of the vocabulary none does, and the probe costs an eighth more.
 template <typename LT, bool VECTOR, int K2_THREADS>
-__device__ int block_inverse_cdf(const LT *a, const LT *d, int V, int mode, float u, float c, float max_a, float sum_a,
+__device__ __forceinline__ int block_inverse_cdf(const LT *a, const LT *d, int V, int mode, float u, float c, float max_a, float sum_a,
                                  float max_b, float sum_b, double approx_total, DrawShared<K2_THREADS / 32> &sh)
 {
     constexpr int VEC = VECTOR ? Logit<LT>::VEC : 1;
     constexpr int NWARP = K2_THREADS / 32;
-    constexpr double guard = 2.0e-5;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    constexpr double guard = 5.0e-6;
     const int nvec = V / VEC;
     const float nma = -max_a * c, nmb = -max_b * c;
     const float ia = 1.0f / sum_a, ib = 1.0f / sum_b;
-    // segments of at least 128 vectors per warp (four 16-byte loads per lane in flight), at most DRAW_MAX_SEG of them
-    int per_warp = 128;
-    {
-        const long long need = ((long long)nvec + DRAW_MAX_SEG - 1) / DRAW_MAX_SEG;
-        const int pw = (int)((need + NWARP - 1) / NWARP);
-        if (pw > per_warp) per_warp = (pw + 31) & ~31;
-    }
-    const int seg_vecs = per_warp * NWARP;
-    const int n_seg = (nvec + seg_vecs - 1) / seg_vecs;
-    const bool early = approx_total > 16.0 * guard;
     const double lo = (double)u * (approx_total - guard), hi = (double)u * (approx_total + guard);
-
-    double running = 0.0, seg_start = 0.0;
-    int s = 0, stop = -1;
-    for (; s < n_seg; ++s) {
-        const int g0 = s * seg_vecs;
-        const int v0 = min(g0 + warp * per_warp, nvec), v1 = min(v0 + per_warp, nvec);
-        const double acc = warp_range_sum<LT, VEC>(a, d, v0, v1, mode, c, nma, ia, nmb, ib);
-        if (lane == 0) sh.tot[s & 1][warp] = acc;
-        __syncthreads();
-        // every warp adds the warps' totals up in the same order
-        double x0 = lane < NWARP ? sh.tot[s & 1][lane] : 0.0;
-        if (NWARP > 32) x0 += lane + 32 < NWARP ? sh.tot[s & 1][lane + 32] : 0.0;
-        const double seg_total = warp_sum(x0);
-        if (tid == 0) sh.seg[s] = seg_total;
-        seg_start = running;
-        running += seg_total;
-        if (early && stop < 0 && running > hi) { stop = s; ++s; break; }
-    }
-    if (stop >= 0 && seg_start <= lo) {
-        // for every total in the band the crossing lies in segment `stop`: find it for the upper end of the band and
-        // take it if the weight in front of it does not reach the lower end
-        const int r0 = stop * seg_vecs, r1 = min(r0 + seg_vecs, nvec);
-        double before;
-        const int tok = locate_in_range<LT, VEC, NWARP>(a, d, r0, r1, mode, c, nma, ia, nmb, ib, seg_start, hi, sh, before);
+    double before, total;
+    const int probe = (nvec / 8 + 31) & ~31;
+    if (approx_total > 16.0 * guard && probe >= NWARP * 32 && probe < nvec) {
+        const int tok = range_inverse_cdf<LT, VEC, NWARP, false>(a, d, probe, mode, hi, c, nma, ia, nmb, ib, sh, before, total);
         if (tok >= 0 && before <= lo) return tok;
-    }
-    // the band did not decide: the rest of the row, then the walk's own total
-    for (; s < n_seg; ++s) {
-        const int g0 = s * seg_vecs;
-        const int v0 = min(g0 + warp * per_warp, nvec), v1 = min(v0 + per_warp, nvec);
-        const double acc = warp_range_sum<LT, VEC>(a, d, v0, v1, mode, c, nma, ia, nmb, ib);
-        if (lane == 0) sh.tot[s & 1][warp] = acc;
         __syncthreads();
-        double x0 = lane < NWARP ? sh.tot[s & 1][lane] : 0.0;
-        if (NWARP > 32) x0 += lane + 32 < NWARP ? sh.tot[s & 1][lane + 32] : 0.0;
-        const double seg_total = warp_sum(x0);
-        if (tid == 0) sh.seg[s] = seg_total;
     }
-    __syncthreads();
-    double threshold = (double)u, base, total;
-    const int sstar = warp_find_part<true>(sh.seg, n_seg, 0.0, threshold, base, total);
-    if (!(total > 0.0)) { __syncthreads(); return -1; }
-    const int r0 = min(sstar * seg_vecs, nvec), r1 = min(r0 + seg_vecs, nvec);
-    double before;
-    return locate_in_range<LT, VEC, NWARP>(a, d, r0, r1, mode, c, nma, ia, nmb, ib, base, threshold, sh, before);
+    return range_inverse_cdf<LT, VEC, NWARP, true>(a, d, nvec, mode, (double)u, c, nma, ia, nmb, ib, sh, before, total);
+}
+
+// The draw from p alone over the whole row, for the one case that needs a second draw: the residual of a rejected
+// position has no mass in fp32 (p == q to rounding).  Rare, so it is a call and not a second inlined copy.
+template <typename LT, bool VECTOR, int K2_THREADS>
+__device__ __noinline__ int draw_from_target(const LT *a, int V, float u, float c, float max_a, float sum_a,
+                                             DrawShared<K2_THREADS / 32> &sh)
+{
+    constexpr int VEC = VECTOR ? Logit<LT>::VEC : 1;
+    double before, total;
+    return range_inverse_cdf<LT, VEC, K2_THREADS / 32, true>(a, nullptr, V / VEC, 2, (double)u, c, -max_a * c, 1.0f / sum_a, 0.f,
+                                                             0.f, sh, before, total);
 }
 
 // Blocks until the kernel launched before this one in the stream has finished and its writes are visible (a no-op
 // when this kernel was launched without programmatic stream serialisation).
 __device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
-// K2_THREADS: the draw walks one row pair per sequence, so a small batch wants large CTAs (many warps keep the
-// load chains short) and a large batch wants many small ones.
+// K2_THREADS: the draw walks (part of) one row pair per sequence, so a small batch wants large CTAs (many warps keep the
+// load chains short) and a large batch wants many small ones.  512 threads per SM in either shape: the draw keeps a
+// dozen fp64 running values next to its loads in flight and wants about 100 registers per thread.
 template <typename LT, bool VECTOR, int K2_THREADS>
 __global__ void __launch_bounds__(K2_THREADS, 1024 / K2_THREADS) epilogue_kernel(const VerifyParams p)
 {
@@ -823,25 +799,26 @@ __global__ void __launch_bounds__(K2_THREADS, 1024 / K2_THREADS) epilogue_kernel
         const double known = mode == 1 ? 1.0 - rs.sum_min : 1.0;
         token = block_inverse_cdf<LT, VECTOR, K2_THREADS>(a, d, V, mode, sh_u, c, rs.max_a, rs.sum_a, rs.max_b, rs.sum_b,
                                                           known, sh_draw);
-        if (token < 0 && mode == 1) {  // p == q in fp32 yet rejected: draw from p
+        if (token < 0 && mode == 1) {  // p == q in fp32 yet rejected (the residual has no mass): draw from p
             __syncthreads();   // every thread has read the first draw's answer before the work space is reused
-            token = block_inverse_cdf<LT, VECTOR, K2_THREADS>(a, nullptr, V, 2, sh_u, c, rs.max_a, rs.sum_a, rs.max_b,
-                                                              rs.sum_b, 1.0, sh_draw);
+            token = draw_from_target<LT, VECTOR, K2_THREADS>(a, V, sh_u, c, rs.max_a, rs.sum_a, sh_draw);
         }
     }
 
-    if (tid == 0) {
+    if (tid < 32) {
+        // the bandit of this sequence: update with the reward, then the next round's arm (one lane per drafter)
         const double r = sh_reward;
-        p.accepted_len[b] = n_acc;
-        p.next_token[b] = token;
-        p.reward[b] = (float)r;
         double *sa = p.st.stat_a + (size_t)b * K, *sb = p.st.stat_b + (size_t)b * K;
         int32_t *wa = p.st.win_arm + (size_t)b * p.tau;
         double *wr = p.st.win_reward + (size_t)b * p.tau;
-        bandit_update(p.bandit, K, p.gamma, p.tau, &p.st.t[b], sa, sb, wa, wr, arm, r);
-        p.st.arm[b] = bandit_select(p.bandit, K, p.beta, p.gamma, p.tau, p.st.t[b], sa, sb, wa, wr, p.seed,
-                                    p.sequence_base + (uint32_t)b);
-        if (sh_flags) atomicOr(p.status, sh_flags);
+        warp_bandit_step(p.bandit, K, p.beta, p.gamma, p.tau, &p.st.t[b], &p.st.arm[b], sa, sb, wa, wr, arm, r, p.seed,
+                         p.sequence_base + (uint32_t)b);
+        if (tid == 0) {
+            p.accepted_len[b] = n_acc;
+            p.next_token[b] = token;
+            p.reward[b] = (float)r;
+            if (sh_flags) atomicOr(p.status, sh_flags);
+        }
     }
 }
 
@@ -924,7 +901,7 @@ static cudaError_t launch_streaming_t(const VerifyParams &p, const RowGeometry &
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     // The epilogue is launched with programmatic stream serialisation: its blocks may be set up while the
     // row-statistics kernel drains, and wait (griddepcontrol.wait) for its completion before they read anything.
-    const bool big_ctas = p.batch <= 320;   // up to about two sequences per SM
+    const bool big_ctas = p.batch <= 320;   // up to about one sequence per SM
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)p.batch);
     cfg.blockDim = dim3(big_ctas ? 512u : 256u);
@@ -953,8 +930,22 @@ cudaError_t launch_streaming(const VerifyParams &p, int dtype, const RowGeometry
 }
 
 // -------------------------------------------------------------------------------------------
-// reset
+// select / reset
 // -------------------------------------------------------------------------------------------
+// The arm of the coming round was chosen at the end of the previous epilogue: selecting is a copy.  (A kernel, not a
+// device-to-device cudaMemcpyAsync: measured on the launch-bound configurations the copy-engine hop cost more.)
+__global__ void select_kernel(const int32_t *arm, int batch, int32_t *arm_out)
+{
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b < batch) arm_out[b] = arm[b];
+}
+
+cudaError_t launch_select(const BanditState &st, int batch, int32_t *arm_out, cudaStream_t stream)
+{
+    select_kernel<<<(batch + 255) / 256, 256, 0, stream>>>(st.arm, batch, arm_out);
+    return cudaGetLastError();
+}
+
 __global__ void reset_kernel(BanditState st, int max_batch, int K, int tau, int variant, double gamma,
                              uint32_t sequence_base, const int32_t *seq_ids, int n)
 {
