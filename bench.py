@@ -73,13 +73,16 @@ def measured_peak_gbs():
 
 def known_traffic(kernel_key: str, workload: str):
     """DRAM bytes (read + write) of one launch of the dominant kernel from the committed ncu capture of exactly this
-    kernel variant on this workload, or None when there is no such capture (a changed kernel has a new key)."""
+    kernel variant on this workload, or None when there is no such capture (a changed variant has another key)."""
     try:
-        with open(os.path.join(ROOT, "profiles", "dram_traffic.json")) as f:
-            table = json.load(f)
-        return table["captures"].get(kernel_key, {}).get(workload)
+        with open(os.path.join(ROOT, "profiles", "dram_traffic.txt")) as f:
+            for line in f:
+                parts = line.split()
+                if len(parts) == 3 and not line.startswith("#") and parts[0] == kernel_key and parts[1] == workload:
+                    return float(parts[2])
     except Exception:
-        return None
+        pass
+    return None
 
 
 class ClockSampler:

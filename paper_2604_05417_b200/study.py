@@ -54,25 +54,32 @@ def both_rewards(res: M.VerifyResult, k: int):
 
 def drafter_reward_statistics(wl: Workload, rounds: int, device=0, seed: int = 0, lib_seed: int = 99) -> List[dict]:
     """Plays every drafter in turn for `rounds` rounds on all sequences (no bandit: the rows are gathered for a
-    fixed drafter index) and returns, per drafter: mean and variance of BD and BE, the share of rounds with BE = 0,
-    the mean accepted length and the mean noise level of that drafter."""
+    fixed drafter index) and returns, per NOISE LEVEL of the drafter (the generator's alignment knob; which drafter
+    has which level differs between sequences and over time): mean and variance of BD and BE, the share of rounds
+    with BE = 0, the mean accepted length and the block efficiency 1 + E[N_acc]."""
     dev = torch.device("cuda", device)
     gen = RoundGenerator(wl, device=dev, seed=seed)
-    rows = []
+    acc: Dict[float, dict] = {}
     for i in range(wl.N):
         msd = M.MetaSD(wl.B, 1, wl.k, wl.V, dtype=wl.dtype, bandit="ucb", device=device)
-        bd, be, zero, sig = RunningMoments(), RunningMoments(), 0, RunningMoments()
         for t in range(rounds):
             rd = gen.gathered_round(t, np.full(wl.B, i))
             res = msd.verify(rd["target"], rd["draft"], rd["tokens"], wl.temperature, lib_seed, want_diag=True)
             r_bd, r_be = both_rewards(res, wl.k)
-            bd.add(r_bd)
-            be.add(r_be)
-            zero += int((r_be == 0).sum())
-            sig.add(rd["sigma"])
+            level = np.round(np.asarray(rd["sigma"], dtype=np.float64), 3)
+            for value in np.unique(level):
+                pick = level == value
+                a = acc.setdefault(float(value), dict(bd=RunningMoments(), be=RunningMoments(), zero=0))
+                a["bd"].add(r_bd[pick])
+                a["be"].add(r_be[pick])
+                a["zero"] += int((r_be[pick] == 0).sum())
         msd.close()
-        rows.append(dict(drafter=i, sigma=sig.mean, mean_bd=bd.mean, var_bd=bd.var, mean_be=be.mean, var_be=be.var,
-                         be_zero_ratio=zero / be.n, mean_accepted=be.mean * wl.k, block_efficiency=1.0 + be.mean * wl.k))
+    rows = []
+    for value in sorted(acc):
+        bd, be = acc[value]["bd"], acc[value]["be"]
+        rows.append(dict(sigma=value, samples=be.n, mean_bd=bd.mean, var_bd=bd.var, mean_be=be.mean, var_be=be.var,
+                         be_zero_ratio=acc[value]["zero"] / be.n, mean_accepted=be.mean * wl.k,
+                         block_efficiency=1.0 + be.mean * wl.k))
     return rows
 
 
@@ -157,7 +164,7 @@ def main():
     report["runs"] = [bandit_run(wl, args.rounds, reward, bandit, window=args.window)
                       for bandit in args.bandits.split(",") for reward in (M.REWARD_BD, M.REWARD_BE)]
     print(json.dumps(report))
-    print(format_table(report["drafters"], ["drafter", "sigma", "mean_bd", "var_bd", "mean_be", "var_be", "be_zero_ratio",
+    print(format_table(report["drafters"], ["sigma", "samples", "mean_bd", "var_bd", "mean_be", "var_be", "be_zero_ratio",
                                             "block_efficiency"]))
     print(format_table(report["runs"], ["bandit", "reward", "best_arm_ratio", "mean_bd", "var_bd", "mean_be", "var_be",
                                         "be_zero_ratio", "block_efficiency"]))
