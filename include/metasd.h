@@ -254,7 +254,8 @@ int metasd_resolved_row_kernel(const metasd_ctx *ctx);
  * and calls no allocating library routine.
  *
  * Runs on the calling thread's current device.  The first call on each device looks up the array's
- * device address (a one-time runtime query): make that first call before any stream capture begins.
+ * device address, and the first call per device and logit type sets the launch attribute its row-statistics
+ * kernel needs (one-time runtime queries, no allocation): make those first calls before any stream capture begins.
  * All calls on a device share the one array and it keeps the previous call's contents; every field
  * the kernels read is rewritten at the start of each call, so calls in stream order are independent,
  * but two calls that overlap on the GPU (different streams, no ordering between them) race on it.
