@@ -826,7 +826,7 @@ __global__ void __launch_bounds__(K2_THREADS, 1024 / K2_THREADS) epilogue_kernel
 // launchers
 // -------------------------------------------------------------------------------------------
 // The built shapes of the staged kernel, per logit type: (threads, stages, CTAs per SM, bonus rows last).
-#define METASD_STAGED_SHAPES(X) X(512, 4, 3, true) X(1024, 6, 1, false) X(1024, 4, 1, true) X(768, 6, 2, true) X(384, 4, 4, true)
+#define METASD_STAGED_SHAPES(X) X(512, 4, 3, true) X(1024, 6, 1, false) X(1024, 4, 1, true) X(768, 4, 2, true) X(384, 4, 4, true)
 
 template <typename LT, int D, int THREADS, int MINB, bool BONUS_LAST>
 static cudaError_t prepare_staged()
