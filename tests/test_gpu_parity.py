@@ -496,6 +496,7 @@ def test_cfg5_full_batch(bandit):
 # ------------------------------------------------------------------------------------------------------------------
 ROW_KERNELS = [dict(row_kernel=M.ROWS_PLAIN), dict(row_kernel=M.ROWS_STAGED),
                dict(row_kernel=M.ROWS_STAGED, row_threads=1024, row_stages=6),
+               dict(row_kernel=M.ROWS_STAGED, row_threads=768, row_stages=4),
                dict(row_kernel=M.ROWS_BULK), dict(row_kernel=M.ROWS_BULK, row_threads=512, row_stages=3),
                dict(row_kernel=M.ROWS_BULK, row_threads=1024, row_stages=7),
                dict(row_kernel=M.ROWS_BULK, row_threads=768, row_stages=8)]
