@@ -53,6 +53,7 @@ def parse_args():
     ap.add_argument("--row-kernel", default="auto", choices=["auto", "plain", "staged", "bulk"])
     ap.add_argument("--row-threads", type=int, default=0)
     ap.add_argument("--row-stages", type=int, default=0)
+    ap.add_argument("--row-cluster", type=int, default=0, help="CTAs that share one row pair (staged row kernel)")
     ap.add_argument("--keep-permille", type=int, default=0)
     ap.add_argument("--order", default="rank", choices=["rank", "reversed", "shuffled"],
                     help="where the likely tokens sit in the vocabulary (the draw walks it in id order)")
@@ -254,7 +255,8 @@ def main():
 
     path = {"auto": M.PATH_AUTO, "streaming": M.PATH_STREAMING, "fused": M.PATH_FUSED}[args.path]
     tuning = dict(row_kernel={"auto": M.ROWS_AUTO, "plain": M.ROWS_PLAIN, "staged": M.ROWS_STAGED, "bulk": M.ROWS_BULK}[args.row_kernel],
-                  row_threads=args.row_threads, row_stages=args.row_stages, keep_permille=args.keep_permille)
+                  row_threads=args.row_threads, row_stages=args.row_stages, keep_permille=args.keep_permille,
+                  row_cluster=args.row_cluster)
     msd = M.MetaSD(wl.B, wl.N, wl.k, wl.V, dtype=wl.dtype, bandit=wl.bandit, beta=wl.beta, gamma=wl.gamma,
                    window=wl.tau, device=local_rank, path=path, sequence_base=rank * wl.B, **tuning)
     path_name = {M.PATH_STREAMING: "streaming", M.PATH_FUSED: "fused"}[msd.resolved_path(wl.k)]
@@ -262,6 +264,8 @@ def main():
     # names the dominant kernel's variant: a capture of DRAM traffic counts only for the variant it was taken on
     kernel_key = path_name if path_name == "fused" else "%s/%s/t%d/s%d/keep%d" % (
         row_kernel, wl.dtype, args.row_threads, args.row_stages, args.keep_permille)
+    if args.row_cluster > 1:
+        kernel_key += "/c%d" % args.row_cluster
 
     # ---- inputs: R distinct rounds, every drafter's logits and tokens resident in HBM
     gen = RoundGenerator(wl, device=dev, seed=1000 + rank)

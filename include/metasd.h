@@ -128,7 +128,8 @@ typedef struct metasd_config {
     int32_t fused_threads;      /* METASD_PATH_FUSED: threads per CTA (0 = chosen from the slice length) */
     int32_t wait_poll_limit;    /* polls after which a device-side wait on an asynchronous copy gives up and sets
                                    METASD_STATUS_TIMEOUT (0 = 2^18 polls of up to 4 us each: about a second).  For tests of that path. */
-    int32_t reserved;           /* must be 0 */
+    int32_t row_cluster;        /* METASD_ROWS_STAGED: CTAs (a thread-block cluster) that share one row pair, each a
+                                   contiguous part of it; 0 or 1 = one CTA per row pair; only the built shapes are accepted */
 } metasd_config;
 
 /* Optional per-position diagnostics of metasd_verify, [B, k]. */

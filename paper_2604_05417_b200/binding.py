@@ -47,7 +47,7 @@ class MetasdConfig(C.Structure):
         ("beta", C.c_double), ("gamma", C.c_double), ("reward_temperature", C.c_double),
         ("row_kernel", C.c_int32), ("row_threads", C.c_int32), ("row_stages", C.c_int32),
         ("keep_permille", C.c_int32), ("fused_cluster", C.c_int32), ("fused_threads", C.c_int32),
-        ("wait_poll_limit", C.c_int32), ("reserved", C.c_int32),
+        ("wait_poll_limit", C.c_int32), ("row_cluster", C.c_int32),
     ]
 
 
@@ -150,7 +150,7 @@ class MetaSD:
                  bandit="ucb", beta: float = 0.01, gamma: float = 0.975, window: int = 50,
                  reward: int = REWARD_BD, reward_temperature: float = 1.0, device: int = 0,
                  path: int = PATH_AUTO, sequence_base: int = 0, host_staging: bool = False, **tuning):
-        """tuning: the configuration's tuning and test fields by name (row_kernel, row_threads, row_stages,
+        """tuning: the configuration's tuning and test fields by name (row_kernel, row_threads, row_stages, row_cluster,
         keep_permille, fused_cluster, fused_threads, wait_poll_limit)."""
         self.lib = load_library()
         cfg = default_config()
@@ -162,7 +162,7 @@ class MetaSD:
         cfg.device, cfg.path, cfg.sequence_base = device, path, sequence_base
         cfg.host_staging = 1 if host_staging else 0
         for name, value in tuning.items():
-            if name not in ("row_kernel", "row_threads", "row_stages", "keep_permille", "fused_cluster",
+            if name not in ("row_kernel", "row_threads", "row_stages", "row_cluster", "keep_permille", "fused_cluster",
                             "fused_threads", "wait_poll_limit"):
                 raise TypeError("unknown configuration field %r" % name)
             setattr(cfg, name, int(value))

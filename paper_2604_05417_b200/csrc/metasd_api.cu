@@ -91,7 +91,7 @@ int validate_config(const metasd_config *c)
     if (c->row_threads < 0 || c->row_stages < 0 || c->keep_permille > 1000) return METASD_ERR_INVALID_ARGUMENT;
     if (c->fused_cluster < 0 || c->fused_cluster > 16 || c->fused_threads < 0 || c->fused_threads % 32 != 0)
         return METASD_ERR_INVALID_ARGUMENT;
-    if (c->wait_poll_limit < 0 || c->reserved != 0) return METASD_ERR_INVALID_ARGUMENT;
+    if (c->wait_poll_limit < 0 || c->row_cluster < 0 || c->row_cluster > 8) return METASD_ERR_INVALID_ARGUMENT;
     if ((uint64_t)c->vocab * (uint64_t)(c->max_draft + 1) >= (1ull << 31)) return METASD_ERR_UNSUPPORTED;
     return METASD_OK;
 }

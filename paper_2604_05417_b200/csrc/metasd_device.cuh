@@ -243,6 +243,9 @@ __device__ __forceinline__ void cluster_sync_all()
     asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
+// The two halves of that barrier on their own (every thread of every CTA of the cluster runs both, in this order).
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
 // Address of the same shared-memory variable in the CTA of the given cluster rank.
 __device__ __forceinline__ uint32_t map_to_rank(uint32_t local, uint32_t rank)
 {

@@ -36,6 +36,7 @@ struct RowGeometry {
     int32_t stages;     // staging depth (0 for plain loads)
     int32_t per_sm;     // CTAs per SM the shape is built for
     int32_t n_sm;       // SMs of the device (persistent kernels size their grid with it)
+    int32_t cluster;    // CTAs that share one row pair (1: none)
 };
 
 struct VerifyParams {

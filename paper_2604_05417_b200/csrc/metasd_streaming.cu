@@ -170,7 +170,12 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, uint64
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-template <typename LT, int D, int THREADS, int MINB, bool BONUS_LAST>
+//
+// CL > 1: a thread-block cluster of CL CTAs shares one row (pair), every CTA a contiguous CL-th of it.  The CTAs
+// exchange their sweep-1 records through distributed shared memory (every CTA gets every record and merges them in
+// rank order, so all hold the same normalisers), sweep their own part again, and rank 0 adds up the parts of
+// sum min(p, q).  The same number of threads then holds a CL-th of the row pairs in flight.
+template <typename LT, int D, int THREADS, int MINB, bool BONUS_LAST, int CL>
 __global__ void __launch_bounds__(THREADS, MINB) row_stats_staged_kernel(const VerifyParams p)
 {
     static_assert(D >= 2, "at least two stages");
@@ -182,21 +187,26 @@ __global__ void __launch_bounds__(THREADS, MINB) row_stats_staged_kernel(const V
     // Blocks are dispatched in index order.  BONUS_LAST: the row pairs come first and the bonus rows (one row, half
     // the work) last, so that the launch ends on its shortest items (measured: better for the bf16 geometry, worse
     // for the fp32 one, which keeps the bonus rows interleaved).
+    const int unit = (int)blockIdx.x / CL;                        // the row (pair) of this CTA or cluster
+    const int rank = CL > 1 ? (int)cluster_rank() : 0;
     const int first_bonus = BONUS_LAST ? p.batch * p.k : 0x7FFFFFFF;
-    const int b = BONUS_LAST ? ((int)blockIdx.x < first_bonus ? (int)blockIdx.x / p.k : (int)blockIdx.x - first_bonus)
-                             : (int)blockIdx.x / (p.k + 1);
+    const int b = BONUS_LAST ? (unit < first_bonus ? unit / p.k : unit - first_bonus) : unit / (p.k + 1);
     const int kb = drafted(p.draft_len, b, p.k);
-    const int j = BONUS_LAST ? ((int)blockIdx.x < first_bonus ? (int)blockIdx.x - b * p.k : kb)
-                             : (int)blockIdx.x - b * (p.k + 1);
+    const int j = BONUS_LAST ? (unit < first_bonus ? unit - b * p.k : kb) : unit - b * (p.k + 1);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const float c = p.c;
     // nothing to do behind the sequence's bonus row; with BONUS_LAST the bonus row belongs to its own late block
-    if (j > kb || (BONUS_LAST && (int)blockIdx.x < first_bonus && j == kb)) return;
+    // (the same for every CTA of a cluster: none of them reaches a cluster barrier)
+    if (j > kb || (BONUS_LAST && unit < first_bonus && j == kb)) return;
     const bool pair = j < kb;
+    // a peer's shared memory may be written once that peer is running: every CTA says so here and checks it after sweep 1
+    if (CL > 1) cluster_arrive();
 
-    const uint4 *a4 = reinterpret_cast<const uint4 *>(reinterpret_cast<const LT *>(p.target) + ((size_t)b * (p.k + 1) + j) * p.V);
-    const uint4 *d4 = pair ? reinterpret_cast<const uint4 *>(draft_rows<LT>(p, b) + ((size_t)b * p.k + j) * p.V) : nullptr;
-    const int nvec = p.V / VEC;
+    const int nvec_row = p.V / VEC;
+    const int v_lo = (int)((long long)nvec_row * rank / CL), v_hi = (int)((long long)nvec_row * (rank + 1) / CL);
+    const uint4 *a4 = reinterpret_cast<const uint4 *>(reinterpret_cast<const LT *>(p.target) + ((size_t)b * (p.k + 1) + j) * p.V) + v_lo;
+    const uint4 *d4 = pair ? reinterpret_cast<const uint4 *>(draft_rows<LT>(p, b) + ((size_t)b * p.k + j) * p.V) + v_lo : nullptr;
+    const int nvec = v_hi - v_lo;   // vectors of this CTA, numbered from 0
     const int n_trip = tid < nvec ? (nvec - tid + THREADS - 1) / THREADS : 0;   // vectors of this thread
     const uint32_t slot0 = smem_addr(stage_mem) + (uint32_t)tid * 16u;
 
@@ -209,7 +219,7 @@ __global__ void __launch_bounds__(THREADS, MINB) row_stats_staged_kernel(const V
     ArgMax am = {METASD_NEG_BIG, 0x7FFFFFFF};
     // a bonus row is read once: nothing of it is worth keeping in L2
     const uint64_t drop = l2_policy_evict_first(), keep = pair ? l2_policy_evict_last() : drop;
-    const int keep_from = p.keep_from_vec;   // first 16-byte vector of a row that L2 is asked to keep (set by the host)
+    const int keep_from = p.keep_from_vec / CL;   // first 16-byte vector of this CTA's part that L2 is asked to keep
     // One group of copies per call, empty past the end: the group count stays in step with the trips.
     auto request1 = [&](int m, int slot, uint64_t pol) {
         if (m < n_trip) {
@@ -241,7 +251,7 @@ __global__ void __launch_bounds__(THREADS, MINB) row_stats_staged_kernel(const V
             for (int e = VEC - 1; e >= 0; --e)
                 if (xa[e] == cm) first = e;
             am.v = cm;
-            am.i = i * VEC + first;
+            am.i = (v_lo + i) * VEC + first;
         }
         const float nma = -sa.m * c;
 #pragma unroll
@@ -275,12 +285,18 @@ __global__ void __launch_bounds__(THREADS, MINB) row_stats_staged_kernel(const V
     for (int u = 0; u < D - 1; ++u)
         if (n + u < n_trip) trip1(n + u, u, keep);
     cp_async_wait<0>();
+    if (CL > 1) cluster_wait();
     sb.m = sa.m;   // the draft row's sum is relative to the target row's maximum
 
     __shared__ MaxSum sh_a[NWARP], sh_b[NWARP];
     __shared__ ArgMax sh_am[NWARP];
     __shared__ double sh_min[NWARP];
     __shared__ float sh_bcast[7];
+
+    // records of the cluster's CTAs, written by their owners: of sweep 1, of a redone draft row, of sweep 2
+    __shared__ float sh_xrec[CL][6];
+    __shared__ float sh_xredo[CL][2];
+    __shared__ double sh_xmin[CL];
 
     sa = warp_merge(sa, c);
     sb = warp_merge(sb, c);
@@ -294,7 +310,30 @@ __global__ void __launch_bounds__(THREADS, MINB) row_stats_staged_kernel(const V
         ra = warp_merge(ra, c);
         rb = warp_merge(rb, c);
         rm = warp_argmax(rm);
-        if (lane == 0) {
+        if (CL > 1) {
+            // lane r hands this CTA's record to the CTA of rank r (every lane holds the merged values)
+            if (lane < CL) {
+                const uint32_t dst = map_to_rank(smem_addr(&sh_xrec[rank][0]), (uint32_t)lane);
+                st_cluster(dst, __float_as_int(ra.m));      st_cluster(dst + 4, __float_as_int(ra.s));
+                st_cluster(dst + 8, __float_as_int(rb.m));  st_cluster(dst + 12, __float_as_int(rb.s));
+                st_cluster(dst + 16, __float_as_int(rm.v)); st_cluster(dst + 20, rm.i);
+            }
+        } else if (lane == 0) {
+            sh_bcast[0] = ra.m; sh_bcast[1] = ra.s; sh_bcast[2] = rb.m; sh_bcast[3] = rb.s;
+            second_sweep_offsets(ra, rb, c, sh_bcast + 4);
+            sh_am[0] = rm;
+        }
+    }
+    if (CL > 1) {
+        cluster_sync_all();   // every CTA's record has arrived in every CTA
+        if (tid == 0) {
+            MaxSum ra = {sh_xrec[0][0], sh_xrec[0][1]}, rb = {sh_xrec[0][2], sh_xrec[0][3]};
+            ArgMax rm = {sh_xrec[0][4], __float_as_int(sh_xrec[0][5])};
+            for (int r = 1; r < CL; ++r) {
+                ra = merge(ra, MaxSum{sh_xrec[r][0], sh_xrec[r][1]}, c);
+                rb = merge(rb, MaxSum{sh_xrec[r][2], sh_xrec[r][3]}, c);
+                rm = better(rm, ArgMax{sh_xrec[r][4], __float_as_int(sh_xrec[r][5])});
+            }
             sh_bcast[0] = ra.m; sh_bcast[1] = ra.s; sh_bcast[2] = rb.m; sh_bcast[3] = rb.s;
             second_sweep_offsets(ra, rb, c, sh_bcast + 4);
             sh_am[0] = rm;
@@ -327,7 +366,22 @@ __global__ void __launch_bounds__(THREADS, MINB) row_stats_staged_kernel(const V
         if (warp == 0) {
             MaxSum rb = lane < NWARP ? sh_b[lane] : MaxSum{METASD_NEG_BIG, 0.f};
             rb = warp_merge(rb, c);
-            if (lane == 0) {
+            if (CL > 1) {
+                if (lane < CL) {
+                    const uint32_t dst = map_to_rank(smem_addr(&sh_xredo[rank][0]), (uint32_t)lane);
+                    st_cluster(dst, __float_as_int(rb.m));
+                    st_cluster(dst + 4, __float_as_int(rb.s));
+                }
+            } else if (lane == 0) {
+                sh_bcast[2] = rb.m; sh_bcast[3] = rb.s;
+                second_sweep_offsets(MaxSum{sh_bcast[0], sh_bcast[1]}, rb, c, sh_bcast + 4);
+            }
+        }
+        if (CL > 1) {
+            cluster_sync_all();   // the verdict above came from the merged records: every CTA of the cluster is here
+            if (tid == 0) {
+                MaxSum rb = {sh_xredo[0][0], sh_xredo[0][1]};
+                for (int r = 1; r < CL; ++r) rb = merge(rb, MaxSum{sh_xredo[r][0], sh_xredo[r][1]}, c);
                 sh_bcast[2] = rb.m; sh_bcast[3] = rb.s;
                 second_sweep_offsets(MaxSum{sh_bcast[0], sh_bcast[1]}, rb, c, sh_bcast + 4);
             }
@@ -377,10 +431,18 @@ __global__ void __launch_bounds__(THREADS, MINB) row_stats_staged_kernel(const V
         __syncthreads();
         if (tid == 0) {
             for (int i = 0; i < NWARP; ++i) total_min += sh_min[i];
+            if (CL > 1) st_cluster(map_to_rank(smem_addr(&sh_xmin[rank]), 0u), total_min);
+        }
+        if (CL > 1) {
+            cluster_sync_all();   // rank 0 holds every part; no CTA leaves while a peer may still write to it
+            if (tid == 0) {
+                total_min = 0.0;
+                for (int r = 0; r < CL; ++r) total_min += sh_xmin[r];
+            }
         }
     }
 
-    if (tid == 0) {
+    if (tid == 0 && rank == 0) {
         RowStats r;
         r.max_a = max_a; r.sum_a = sum_a; r.max_b = max_b; r.sum_b = sum_b;
         r.argmax_a = sh_am[0].i;
@@ -394,12 +456,25 @@ __global__ void __launch_bounds__(THREADS, MINB) row_stats_staged_kernel(const V
     }
 }
 
-template <typename LT, int D, int THREADS, int MINB, bool BONUS_LAST>
-static cudaError_t launch_staged(const VerifyParams &p, dim3 grid, cudaStream_t stream)
+template <typename LT, int D, int THREADS, int MINB, bool BONUS_LAST, int CL>
+static cudaError_t launch_staged(const VerifyParams &p, unsigned units, cudaStream_t stream)
 {
     const size_t smem = (size_t)D * 2 * THREADS * 16;   // the attribute that allows it was set by streaming_prepare
-    row_stats_staged_kernel<LT, D, THREADS, MINB, BONUS_LAST><<<grid, THREADS, smem, stream>>>(p);
-    return cudaSuccess;
+    if (CL == 1) {
+        row_stats_staged_kernel<LT, D, THREADS, MINB, BONUS_LAST, CL><<<units, THREADS, smem, stream>>>(p);
+        return cudaSuccess;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(units * CL);
+    cfg.blockDim = dim3(THREADS);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute at;
+    at.id = cudaLaunchAttributeClusterDimension;
+    at.val.clusterDim.x = CL; at.val.clusterDim.y = 1; at.val.clusterDim.z = 1;
+    cfg.attrs = &at;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, row_stats_staged_kernel<LT, D, THREADS, MINB, BONUS_LAST, CL>, p);
 }
 
 // -------------------------------------------------------------------------------------------
@@ -825,20 +900,22 @@ __global__ void __launch_bounds__(K2_THREADS, 1024 / K2_THREADS) epilogue_kernel
 // -------------------------------------------------------------------------------------------
 // launchers
 // -------------------------------------------------------------------------------------------
-// The built shapes of the staged kernel, per logit type: (threads, stages, CTAs per SM, bonus rows last).
-#define METASD_STAGED_SHAPES(X) X(512, 4, 3, true) X(1024, 6, 1, false) X(1024, 4, 1, true) X(768, 4, 2, true) X(384, 4, 4, true)
+// The built shapes of the staged kernel, per logit type: (threads, stages, CTAs per SM, bonus rows last, CTAs per row).
+#define METASD_STAGED_SHAPES(X) \
+    X(512, 4, 3, true, 1) X(1024, 6, 1, false, 1) X(1024, 4, 1, true, 1) X(768, 4, 2, true, 1) X(384, 4, 4, true, 1) \
+    X(512, 4, 3, true, 3) X(512, 4, 3, true, 2) X(768, 4, 2, true, 2)
 
-template <typename LT, int D, int THREADS, int MINB, bool BONUS_LAST>
+template <typename LT, int D, int THREADS, int MINB, bool BONUS_LAST, int CL>
 static cudaError_t prepare_staged()
 {
-    return cudaFuncSetAttribute(row_stats_staged_kernel<LT, D, THREADS, MINB, BONUS_LAST>,
+    return cudaFuncSetAttribute(row_stats_staged_kernel<LT, D, THREADS, MINB, BONUS_LAST, CL>,
                                 cudaFuncAttributeMaxDynamicSharedMemorySize, D * 2 * THREADS * 16);
 }
 
 template <typename LT>
-static cudaError_t prepare_staged_t(int threads, int stages, int *per_sm)
+static cudaError_t prepare_staged_t(int threads, int stages, int cluster, int *per_sm)
 {
-#define X(T, D, M, BL) if (threads == T && stages == D) { *per_sm = M; return prepare_staged<LT, D, T, M, BL>(); }
+#define X(T, D, M, BL, C) if (threads == T && stages == D && cluster == C) { *per_sm = M; return prepare_staged<LT, D, T, M, BL, C>(); }
     METASD_STAGED_SHAPES(X)
 #undef X
     return cudaErrorNotSupported;
@@ -847,8 +924,8 @@ static cudaError_t prepare_staged_t(int threads, int stages, int *per_sm)
 template <typename LT>
 static cudaError_t launch_staged_t(const VerifyParams &p, const RowGeometry &geo, cudaStream_t stream)
 {
-    const dim3 grid((unsigned)p.batch * (unsigned)(p.k + 1));
-#define X(T, D, M, BL) if (geo.threads == T && geo.stages == D) return launch_staged<LT, D, T, M, BL>(p, grid, stream);
+    const unsigned units = (unsigned)p.batch * (unsigned)(p.k + 1);
+#define X(T, D, M, BL, C) if (geo.threads == T && geo.stages == D && geo.cluster == C) return launch_staged<LT, D, T, M, BL, C>(p, units, stream);
     METASD_STAGED_SHAPES(X)
 #undef X
     return cudaErrorNotSupported;
@@ -865,6 +942,7 @@ cudaError_t streaming_prepare(int device, int dtype, const metasd_config &cfg, R
     geo->threads = cfg.row_threads;
     geo->stages = cfg.row_stages;
     geo->per_sm = 1;
+    geo->cluster = 1;
     if (geo->kernel == METASD_ROWS_PLAIN) {
         if (geo->threads && geo->threads != K1_THREADS) return cudaErrorNotSupported;
         geo->threads = K1_THREADS;
@@ -880,8 +958,9 @@ cudaError_t streaming_prepare(int device, int dtype, const metasd_config &cfg, R
     if (geo->kernel != METASD_ROWS_STAGED) return cudaErrorNotSupported;
     if (!geo->threads) geo->threads = dtype == METASD_BF16 ? 512 : 1024;
     if (!geo->stages) geo->stages = dtype == METASD_BF16 ? 4 : 6;
-    return dtype == METASD_BF16 ? prepare_staged_t<__nv_bfloat16>(geo->threads, geo->stages, &geo->per_sm)
-                                : prepare_staged_t<float>(geo->threads, geo->stages, &geo->per_sm);
+    geo->cluster = cfg.row_cluster > 1 ? cfg.row_cluster : 1;
+    return dtype == METASD_BF16 ? prepare_staged_t<__nv_bfloat16>(geo->threads, geo->stages, geo->cluster, &geo->per_sm)
+                                : prepare_staged_t<float>(geo->threads, geo->stages, geo->cluster, &geo->per_sm);
 }
 
 template <typename LT>

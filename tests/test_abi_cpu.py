@@ -53,7 +53,7 @@ def test_host_side_validation(lib):
         assert ctx.value is None
     assert all(code == M.ERR_INVALID_ARGUMENT for _, code in bad), bad
     for field, value in [("row_threads", -1), ("keep_permille", 1001), ("fused_cluster", 17), ("fused_threads", 33),
-                         ("wait_poll_limit", -1), ("reserved", 1)]:
+                         ("wait_poll_limit", -1), ("row_cluster", -1), ("row_cluster", 9)]:
         cfg = M.default_config()
         setattr(cfg, field, value)
         assert lib.metasd_init(C.byref(ctx), C.byref(cfg)) == M.ERR_INVALID_ARGUMENT, field

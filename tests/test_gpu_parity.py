@@ -497,6 +497,9 @@ def test_cfg5_full_batch(bandit):
 ROW_KERNELS = [dict(row_kernel=M.ROWS_PLAIN), dict(row_kernel=M.ROWS_STAGED),
                dict(row_kernel=M.ROWS_STAGED, row_threads=1024, row_stages=6),
                dict(row_kernel=M.ROWS_STAGED, row_threads=768, row_stages=4),
+               dict(row_kernel=M.ROWS_STAGED, row_threads=512, row_stages=4, row_cluster=3),
+               dict(row_kernel=M.ROWS_STAGED, row_threads=768, row_stages=4, row_cluster=2),
+               dict(row_kernel=M.ROWS_STAGED, row_threads=512, row_stages=4, row_cluster=2),
                dict(row_kernel=M.ROWS_BULK), dict(row_kernel=M.ROWS_BULK, row_threads=512, row_stages=3),
                dict(row_kernel=M.ROWS_BULK, row_threads=1024, row_stages=7),
                dict(row_kernel=M.ROWS_BULK, row_threads=768, row_stages=8)]
@@ -516,8 +519,9 @@ def test_row_kernel_variants(tuning, dtype, V, T):
         assert c["near_tie_accept"] == 0 and c["near_tie_token"] == 0 and c["near_tie_arm"] == 0
 
 
-@pytest.mark.parametrize("tuning", [dict(row_kernel=M.ROWS_STAGED), dict(row_kernel=M.ROWS_BULK)],
-                         ids=["staged", "bulk"])
+@pytest.mark.parametrize("tuning", [dict(row_kernel=M.ROWS_STAGED), dict(row_kernel=M.ROWS_BULK),
+                                    dict(row_kernel=M.ROWS_STAGED, row_threads=512, row_stages=4, row_cluster=3)],
+                         ids=["staged", "bulk", "staged-cluster3"])
 def test_row_kernels_with_per_sequence_draft_lengths_and_odd_logit_scales(tuning):
     """The bulk-copy kernel skips positions behind a sequence's draft length and redoes a draft row whose sum the
     shared reference flushed, like the staged kernel does."""
