@@ -943,6 +943,7 @@ cudaError_t streaming_prepare(int device, int dtype, const metasd_config &cfg, R
     geo->stages = cfg.row_stages;
     geo->per_sm = 1;
     geo->cluster = 1;
+    if (cfg.row_cluster > 1 && geo->kernel != METASD_ROWS_STAGED) return cudaErrorNotSupported;   // only the staged kernel has a cluster form
     if (geo->kernel == METASD_ROWS_PLAIN) {
         if (geo->threads && geo->threads != K1_THREADS) return cudaErrorNotSupported;
         geo->threads = K1_THREADS;

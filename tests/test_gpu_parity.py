@@ -235,6 +235,17 @@ def test_fused_path_declines_per_sequence_draft_lengths():
         gpu.close()
 
 
+@pytest.mark.parametrize("tuning", [dict(row_kernel=M.ROWS_STAGED, row_threads=640), dict(row_kernel=M.ROWS_STAGED, row_stages=5),
+                                    dict(row_kernel=M.ROWS_STAGED, row_cluster=4), dict(row_kernel=M.ROWS_BULK, row_cluster=2),
+                                    dict(row_kernel=M.ROWS_PLAIN, row_cluster=2), dict(row_kernel=M.ROWS_BULK, row_stages=9)],
+                         ids=lambda d: "-".join("%s%s" % kv for kv in d.items()))
+def test_a_row_kernel_shape_that_is_not_built_is_declined_at_init(tuning):
+    """Only the built shapes of the row-statistics kernels are accepted; anything else is UNSUPPORTED, not a fallback."""
+    with pytest.raises(M.MetasdError) as err:
+        M.MetaSD(4, 2, 3, 4096, dtype="bf16", device=0, **tuning)
+    assert err.value.code == M.ERR_UNSUPPORTED
+
+
 @pytest.mark.parametrize("dtype", ["bf16", "fp32"])
 @pytest.mark.parametrize("T", [1.0, 0.5])
 def test_draft_rows_on_another_scale_than_the_target(dtype, T):
