@@ -2,7 +2,8 @@
 
 The paper compares its two alignment rewards on real drafters: their means and variances, how often BE is exactly
 zero, and how quickly a bandit fed with either reward settles on the best drafter (Sec. 2.3: the BE definition and
-the lemma that relates E[r^BE] to E[r^BD]; the reward-statistics table; the best-arm-ratio figure).  This module
+the lemma that relates E[r^BE] to E[r^BD]; Theorem 1's feedback signal; the reward-statistics table; the best-arm-ratio
+figure).  This module
 produces the same quantities for the synthetic workloads, whose generator knows which drafter is best for every
 sequence in every round.  Every round runs through the library (C ABI, CUDA kernels); what is computed here is
 bookkeeping on its outputs: means, variances, counts.
@@ -80,6 +81,29 @@ def drafter_reward_statistics(wl: Workload, rounds: int, device=0, seed: int = 0
         rows.append(dict(sigma=value, samples=be.n, mean_bd=bd.mean, var_bd=bd.var, mean_be=be.mean, var_be=be.var,
                          be_zero_ratio=acc[value]["zero"] / be.n, mean_accepted=be.mean * wl.k,
                          block_efficiency=1.0 + be.mean * wl.k))
+    return add_feedback_signal(rows)
+
+
+def feedback_signal(mean_best: float, var_best: float, mean_i: float, var_i: float) -> float:
+    """The bandit feedback signal of a suboptimal drafter i under one reward design (the equation of Theorem 1):
+    R = Delta_i^2 / max(Var[r_i], Var[r_best]) with Delta_i = mu_best - mu_i.  Infinite when neither reward varies."""
+    gap, spread = mean_best - mean_i, max(var_i, var_best)
+    if spread > 0.0:
+        return gap * gap / spread
+    return float("inf") if gap != 0.0 else float("nan")
+
+
+def add_feedback_signal(rows: List[dict]) -> List[dict]:
+    """Adds `signal_bd` and `signal_be` to the rows of drafter_reward_statistics: the feedback signal of every
+    drafter against the best one, which is the row with the smallest noise level (the generator's best drafter;
+    its own signal is NaN)."""
+    best = min(rows, key=lambda r: r["sigma"])
+    for r in rows:
+        if r is best:
+            r["signal_bd"] = r["signal_be"] = float("nan")
+        else:
+            r["signal_bd"] = feedback_signal(best["mean_bd"], best["var_bd"], r["mean_bd"], r["var_bd"])
+            r["signal_be"] = feedback_signal(best["mean_be"], best["var_be"], r["mean_be"], r["var_be"])
     return rows
 
 
@@ -165,7 +189,7 @@ def main():
                       for bandit in args.bandits.split(",") for reward in (M.REWARD_BD, M.REWARD_BE)]
     print(json.dumps(report))
     print(format_table(report["drafters"], ["sigma", "samples", "mean_bd", "var_bd", "mean_be", "var_be", "be_zero_ratio",
-                                            "block_efficiency"]))
+                                            "block_efficiency", "signal_bd", "signal_be"]))
     print(format_table(report["runs"], ["bandit", "reward", "best_arm_ratio", "mean_bd", "var_bd", "mean_be", "var_be",
                                         "be_zero_ratio", "block_efficiency"]))
     for r in report["runs"]:

@@ -80,3 +80,5 @@ def test_best_arm_ratio_and_histogram_of_a_short_bandit_run():
     assert 0 < out["mean_bd"] <= 1 and 1.0 <= out["block_efficiency"] <= wl.k + 1
     rows = study.drafter_reward_statistics(wl, rounds=2)
     assert len(rows) == wl.N and all(r["var_be"] >= 0 for r in rows)
+    # Theorem 1's feedback signal of every drafter against the best (the smallest noise level): BD's is the stronger
+    assert np.isnan(rows[0]["signal_bd"]) and all(r["signal_bd"] > r["signal_be"] > 0 for r in rows[1:])

@@ -46,6 +46,32 @@ def test_running_moments_and_table_format():
     assert text.splitlines()[0] == "| a | b |" and text.splitlines()[-1] == "| 1 | 0.5000 |"
 
 
+def test_feedback_signal_on_the_papers_reward_statistics_table():
+    """Theorem 1's feedback signal R = Delta^2 / max(Var[r_i], Var[r_best]) evaluated on the statistics the paper prints
+    for its five drafters: BD gives every suboptimal drafter the stronger signal, which is the paper's reading of that
+    table.  The two figures for the Russian drafter are worked out by hand from the printed numbers:
+    BD (0.488 - 0.294)^2 / 0.044 = 0.855, BE (0.232 - 0.099)^2 / 0.093 = 0.190."""
+    import os
+    from paper_2604_05417_b200 import study
+    rows = []
+    with open(os.path.join(os.path.dirname(__file__), "golden", "reward_statistics_table.txt")) as f:
+        for line in f:
+            if line.startswith("#") or not line.strip():
+                continue
+            name, mean_be, mean_bd, var_be, var_bd, zero = line.split()
+            # the study's rows are keyed by noise level, smallest = best: give the best drafter (first line) level 0
+            rows.append(dict(name=name, sigma=float(len(rows)), mean_be=float(mean_be), mean_bd=float(mean_bd),
+                             var_be=float(var_be), var_bd=float(var_bd)))
+    rows = study.add_feedback_signal(rows)
+    assert rows[0]["name"] == "Ja" and np.isnan(rows[0]["signal_bd"]) and np.isnan(rows[0]["signal_be"])
+    assert all(r["signal_bd"] > r["signal_be"] > 0 for r in rows[1:])
+    ru = rows[1]
+    assert abs(ru["signal_bd"] - 0.855) < 1e-3 and abs(ru["signal_be"] - 0.190) < 1e-3
+    assert study.feedback_signal(0.5, 0.0, 0.25, 0.0) == float("inf")          # rewards that do not vary
+    # the larger of the two variances counts, whichever drafter it belongs to
+    assert study.feedback_signal(0.5, 0.01, 0.3, 0.04) == study.feedback_signal(0.5, 0.04, 0.3, 0.01) == 0.2 ** 2 / 0.04
+
+
 def test_constant_alignment_rows_have_the_prescribed_alignment():
     """The rows of the reward pins: 1 - d_TV(p_j, q_j) is the requested alpha, and the drafted token is the drafter's
     only token (float64 softmax of the generated logits, typed out here)."""
