@@ -55,6 +55,8 @@ def parse_args():
     ap.add_argument("--row-stages", type=int, default=0)
     ap.add_argument("--row-cluster", type=int, default=0, help="CTAs that share one row pair (staged row kernel)")
     ap.add_argument("--keep-permille", type=int, default=0)
+    ap.add_argument("--graph", action="store_true",
+                    help="capture every step (select + verify) into a CUDA graph before the timed region and replay it there")
     ap.add_argument("--order", default="rank", choices=["rank", "reversed", "shuffled"],
                     help="where the likely tokens sit in the vocabulary (the draw walks it in id order)")
     ap.add_argument("--sustained-seconds", type=float, default=1.0,
@@ -288,11 +290,27 @@ def main():
     rew_all = torch.zeros((n_all, wl.B), dtype=torch.float32, device=dev)   # timed region
     outs = [M.VerifyResult(acc_all[i], tok_all[i], rew_all[i]) for i in range(n_all)]
 
-    def step(i):
+    def launch_step(i):
         rd = rounds[i % len(rounds)]
         msd.select(out=arm_buf)
         msd.verify(rd["target"], None, rd["tokens"], wl.temperature, LIB_SEED, drafter_table=rd["table"],
                    token_arm_stride=stride, out=outs[i])
+
+    step, graphs = launch_step, []
+    if args.graph:
+        # neither call allocates or synchronises and the round counter lives in the device state, so a captured step
+        # replays as the next round; one graph per step because every step writes its own output slice
+        side = torch.cuda.Stream(device=dev)
+        side.wait_stream(torch.cuda.current_stream(dev))
+        before = msd.kernel_launches()
+        for i in range(n_all):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                launch_step(i)
+            graphs.append(g)
+        torch.cuda.synchronize()
+        launches_per_step = (msd.kernel_launches() - before) // n_all
+        step = lambda i: graphs[i].replay()
 
     def barrier():
         if world > 1:
@@ -318,7 +336,7 @@ def main():
     t_end.record()
     barrier()
     host_end = time.time()
-    launches = msd.kernel_launches() - launches0
+    launches = launches_per_step * args.steps if args.graph else msd.kernel_launches() - launches0
     # ---- a timed region under half a second says little about sustained rounds (the power cap acts after a few
     # hundred milliseconds): run an extra leg of back-to-back rounds and report it beside the timed one
     sustained = None
@@ -377,7 +395,7 @@ def main():
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": wl.name, "B_per_gpu": wl.B, "N": wl.N, "k": wl.k, "V": wl.V, "logits": wl.dtype,
                    "temperature": wl.temperature, "bandit": wl.bandit, "path": path_name, "row_kernel": row_kernel,
-                   "vocab_order": wl.order,
+                   "vocab_order": wl.order, "launch": "cuda graph replay, one graph per step" if args.graph else "stream launches",
                    "draft_len": "uniform 1..k per sequence" if args.ragged else "k for every sequence",
                    "l2": "inputs larger than L2: %.2f GB read per step, %d rotating input sets" % (bytes_round / 1e9, len(rounds))},
         "rounds_per_s": world * args.steps / (total_ms * 1e-3),

@@ -20,6 +20,9 @@
  *     state and its scratch; nothing is allocated after metasd_init.
  *   - Calls are asynchronous on the CUDA stream passed as `stream` (a cudaStream_t, typed void*
  *     so that this header needs no CUDA include); calls on one context must be stream-ordered.
+ *     metasd_select, metasd_verify and metasd_reset only launch kernels: they may be captured into
+ *     a CUDA graph.  A replay is the context's next round on whatever the captured buffers then
+ *     hold (the round counter that keys the random numbers is device state, not a launch argument).
  *   - A context belongs to the device named in its configuration.  Every call that takes a context
  *     makes that device current for its own duration and restores the caller's current device before
  *     it returns; `stream` must be a stream of the context's device (or NULL).

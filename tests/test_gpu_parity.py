@@ -624,3 +624,55 @@ def test_context_calls_run_on_the_contexts_device_and_leave_the_callers_current_
     gpu.select()
     assert torch.cuda.current_device() == before
     gpu.close()
+
+
+# ------------------------------------------------------------------------------------------------------------------
+# Replay from a CUDA graph
+# ------------------------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("dtype,T", [("bf16", 0.0), ("fp32", 1.0)])
+def test_select_and_verify_replayed_from_a_cuda_graph(dtype, T):
+    """metasd_select + metasd_verify neither allocate nor synchronise, and the round counter that keys the random
+    numbers lives in the device state: one captured round, replayed on buffers that are refilled in place, gives the
+    oracle's rounds one after the other (pointer-table mode, so the bandit's own choice picks the rows)."""
+    from _harness import make_pair, compare_round, gather_by_arm
+    wl = base(B=12, N=3, k=4, V=16384, sigmas=(0.3, 1.0, 2.5)).scaled(dtype=dtype, temperature=T)
+    dev = torch.device("cuda", 0)
+    gen = RoundGenerator(wl, device=dev, seed=17)
+    gpu, orc = make_pair(wl, path=M.PATH_STREAMING)
+    first = gen.table_round(0)
+    target, tokens = first["target"].clone(), first["tokens"].clone()
+    drafts = [d.clone() for d in first["drafts"]]
+    table = M.pointer_table(drafts)
+    arm_out = torch.empty(wl.B, dtype=torch.int32, device=dev)
+    res = M.VerifyResult(torch.empty(wl.B, dtype=torch.int32, device=dev), torch.empty(wl.B, dtype=torch.int32, device=dev),
+                         torch.empty(wl.B, dtype=torch.float32, device=dev))
+    res.diag = torch.zeros((wl.B, wl.k, 5), dtype=torch.float32, device=dev)
+    counts = {"sequences": wl.B, "near_tie_accept": 0, "near_tie_token": 0, "near_tie_arm": 0}
+    try:
+        launches_before = gpu.kernel_launches()
+        graph = torch.cuda.CUDAGraph()
+        side = torch.cuda.Stream(device=dev)
+        side.wait_stream(torch.cuda.current_stream(dev))
+        with torch.cuda.graph(graph, stream=side):
+            gpu.select(out=arm_out)
+            gpu.verify(target, None, tokens, T, 77, drafter_table=table, token_arm_stride=wl.B * wl.k, out=res)
+        torch.cuda.synchronize()
+        assert M.parse_state(gpu.state_export(), wl.B, wl.N, wl.tau)["t"].max() == 0, "capturing does not run the round"
+        assert gpu.kernel_launches() - launches_before == 3      # select, row statistics, epilogue: the captured round
+        for t in range(7):
+            rd = gen.table_round(t)
+            target.copy_(rd["target"]); tokens.copy_(rd["tokens"])
+            for dst, src in zip(drafts, rd["drafts"]):
+                dst.copy_(src)
+            graph.replay()
+            torch.cuda.synchronize()
+            arm_o = orc.select()
+            assert np.array_equal(arm_out.cpu().numpy(), arm_o)
+            draft, tok = gather_by_arm(rd["drafts"], rd["tokens"], arm_o, dev)
+            out = orc.verify(rd["target"], None, tok.cpu().numpy(), T, 77, drafter_tables=rd["drafts"])
+            out["_reward_kind"] = M.REWARD_BD
+            compare_round(res, out, rd["target"], draft, T, 1.0, counts)
+        assert gpu.last_status() == 0
+        assert np.array_equal(M.parse_state(gpu.state_export(), wl.B, wl.N, wl.tau)["t"], orc.t)
+    finally:
+        gpu.close()
